@@ -1,0 +1,157 @@
+/*
+ * opt_tree.h — C ABI of the B200 (sm_100a) OPT-Tree draft-tree library.
+ *
+ * One decoding step of speculative decoding with an adaptive draft tree (Algorithm 2 of
+ * the OPT-Tree paper) is: construct the tree (Algorithm 1), compute its tree attention
+ * mask, run the target model on it, verify.  This library implements everything in that
+ * step except the two model forwards, which are replaced by bf16 logit tables:
+ *
+ *   draft "model"  L_d [H][V] bf16, target "model" L_t [H][V] bf16, row-major; the next-token
+ *   logits of a node holding token t at depth d (root: d = 0) are row (t*31 + d) mod H.
+ *
+ * Conventions
+ *   - Every pointer marked (dev) is device memory on the context's device, owned by the
+ *     caller; (host) is host memory.  build / mask / verify / row_softmax_topk only enqueue
+ *     work on `stream` (a cudaStream_t passed as void*, NULL = default stream); they never
+ *     allocate, free or synchronise.
+ *   - Return value: OPT_TREE_OK (0) or a negative opt_tree_status.  Nothing throws, aborts
+ *     or traps.  Errors detected on the device (a bounded wait that expired, an index that
+ *     failed its bounds check) are recorded in a device status word, read back with
+ *     opt_tree_last_device_status().
+ *   - Logits must be finite or -inf (no NaN, no +inf); a row must hold at least one finite
+ *     value.  Behaviour on other inputs is unspecified but never faults.
+ *   - The root is not a node of the output, is not counted in n and has no mask bit
+ *     (Section 3: "the root node is not considered when calculating node trees").
+ */
+#ifndef OPT_TREE_H_
+#define OPT_TREE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    OPT_TREE_OK = 0,
+    OPT_TREE_ERR_INVALID_ARG = -1,   /* null pointer, non-positive size, B > max_batch ... */
+    OPT_TREE_ERR_UNSUPPORTED = -2,   /* n > 256, k > 32, k > V, misaligned table ... */
+    OPT_TREE_ERR_CUDA = -3,          /* a CUDA runtime call failed */
+    OPT_TREE_ERR_TIMEOUT = -4,       /* a bounded device-side wait expired */
+    OPT_TREE_ERR_INTERNAL = -5       /* a device-side bounds check failed */
+} opt_tree_status;
+
+#define OPT_TREE_MAX_N 256
+#define OPT_TREE_MAX_K 32
+
+typedef struct opt_tree_ctx opt_tree_ctx;   /* opaque; owns only its workspace */
+
+/* Problem sizes fixed for the lifetime of a context.
+ *   V          vocabulary size (columns of the tables), V >= 1
+ *   H          rows of the tables, H >= 1
+ *   n          node budget of the tree (Algorithm 1 input n), 1 <= n <= OPT_TREE_MAX_N
+ *   k          at most k children per node (the k most probable next tokens), 1 <= k <= OPT_TREE_MAX_K
+ *   max_depth  cap on the number of drafted layers; Algorithm 1 also caps the depth by n
+ *   max_batch  largest B any call will pass */
+typedef struct {
+    int32_t V, H, n, k, max_depth, max_batch;
+} opt_tree_config;
+
+/* One batch of built trees, structure of arrays (all dev).  Nodes of a tree are packed in
+ * the order (depth ascending, parent's packed index ascending, sibling rank ascending), so a
+ * parent always precedes its children.  Unused tail slots i >= n_sel hold token -1,
+ * parent -1, depth 0, phat 0. */
+typedef struct {
+    int32_t *token;          /* [B][n]  token id of node i */
+    int32_t *parent;         /* [B][n]  packed index of the parent, -1 = child of the root */
+    int32_t *depth;          /* [B][n]  1-based depth */
+    double  *phat;           /* [B][n]  path value, Eq. 2: product of draft probabilities along the path */
+    int32_t *n_sel;          /* [B]     nodes kept, min(n, nodes drafted) */
+    int32_t *depth_reached;  /* [B]     layers drafted before the loop of Algorithm 1 stopped */
+    double  *expected_len;   /* [B]     E(A), Eq. 3: sum of the kept path values */
+    double  *esub_trace;     /* [B][max_depth] or NULL: E_sub(T, n) after each drafted layer, 0 beyond */
+} opt_tree_out;
+
+/* Workspace bytes a context allocates for cfg (0 if cfg is invalid). */
+size_t opt_tree_workspace_bytes(const opt_tree_config *cfg);
+
+/* Creates a context on the current CUDA device and allocates its workspace once
+ * (cudaMalloc).  *ctx is set to NULL on failure. */
+int opt_tree_create(opt_tree_ctx **ctx, const opt_tree_config *cfg);
+int opt_tree_destroy(opt_tree_ctx *ctx);
+
+/* Algorithm 1 ("Construct an OPT-Tree") for B independent sequences.
+ *   draft_logits_bf16 (dev) [H][V]   16-byte aligned base
+ *   root_token        (dev) [B]      last token x_l of each input sequence, 0 <= token < V
+ *   delta                            threshold of the loop test (E_sub(T,n) - E > delta); pass
+ *                                    -INFINITY to draft min(max_depth, n) layers unconditionally
+ *   out                              filled as described at opt_tree_out
+ * Per layer, every node of the last layer is expanded (fused row softmax + top-k over V), the
+ * candidates' path values are parent value x child probability (Eq. 2), the next layer is the n
+ * candidates of largest path value (ties: lower candidate index), E_sub(T,n) is the sum of the n
+ * largest path values drafted so far, and the final tree is those n nodes (last line of
+ * Algorithm 1).  The layer whose gain did not exceed delta stays in T. */
+int opt_tree_build(opt_tree_ctx *ctx, const void *draft_logits_bf16, const int32_t *root_token,
+                   int32_t B, float delta, const opt_tree_out *out, void *stream);
+
+/* Tree attention mask and position ids (Algorithm 2, second line; Figure 1 caption: nodes of
+ * one layer share a position index).
+ *   tree          a batch written by opt_tree_build (parent, depth, n_sel are read)
+ *   base_pos      (dev) [B] or NULL (= 0): position of the root token
+ *   mask          (dev) [B][n][W], W = ceil(n/64): bit (j % 64) of word j/64 of row i is set iff
+ *                 node j is node i or an ancestor of node i; rows i >= n_sel are zero.  The root
+ *                 and the prefix are visible to every node and are not stored.
+ *   position_ids  (dev) [B][n]: base_pos + depth for kept nodes, 0 for unused slots */
+int opt_tree_mask(opt_tree_ctx *ctx, const opt_tree_out *tree, int32_t B, const int32_t *base_pos,
+                  uint64_t *mask, int32_t *position_ids, void *stream);
+
+/* Greedy verification (Preliminaries, greedy sampling; Algorithm 2, Verify): the target's
+ * most probable token after the root and after every kept node (ties: lowest token id), then
+ * the longest root branch that follows those tokens, plus the token after the last hit.
+ *   target_logits_bf16 (dev) [H][V]
+ *   accept_len    (dev) [B]               A = matched nodes + 1  (1 <= A <= depth_reached + 1)
+ *   accept_tokens (dev) [B][max_depth+1]  the A accepted tokens, then -1
+ *   accept_nodes  (dev) [B][max_depth]    packed indices of the A-1 matched nodes, then -1
+ *   next_root     (dev) [B]               last accepted token = root of the next step */
+int opt_tree_verify(opt_tree_ctx *ctx, const opt_tree_out *tree, const void *target_logits_bf16,
+                    const int32_t *root_token, int32_t B, int32_t *accept_len, int32_t *accept_tokens,
+                    int32_t *accept_nodes, int32_t *next_root, void *stream);
+
+/* The row step of Algorithm 1 on its own (children rule after Eq. 2): for each listed row,
+ * the min(k, V) most probable tokens (logit descending, token id ascending) and their softmax
+ * probabilities.
+ *   logits_bf16 (dev) [H][V];  rows (dev) [nrows] row indices in [0, H)
+ *   tok_out (dev) [nrows][k] int32, prob_out (dev) [nrows][k] double (entries >= min(k,V): -1 / 0) */
+int opt_tree_row_softmax_topk(opt_tree_ctx *ctx, const void *logits_bf16, const int32_t *rows,
+                              int32_t nrows, int32_t *tok_out, double *prob_out, void *stream);
+
+/* One whole decoding step (build, mask, verify) with HOST buffers: copies root_token and
+ * base_pos to the device, runs the three stages, copies every output back and synchronises the
+ * stream before returning.  The logit tables stay on the device (they stand in for the models).
+ * Host buffers should be pinned for the copies to be asynchronous.  Any output pointer may be
+ * NULL to skip its copy; shapes are those of opt_tree_out / opt_tree_mask / opt_tree_verify. */
+typedef struct {
+    int32_t *token, *parent, *depth; double *phat;                 /* (host) [B][n] */
+    int32_t *n_sel, *depth_reached; double *expected_len;          /* (host) [B] */
+    uint64_t *mask; int32_t *position_ids;                         /* (host) [B][n][W], [B][n] */
+    int32_t *accept_len, *accept_tokens, *accept_nodes, *next_root;/* (host) [B], [B][D+1], [B][D], [B] */
+} opt_tree_host_out;
+
+int opt_tree_step_host(opt_tree_ctx *ctx, const void *draft_logits_bf16, const void *target_logits_bf16,
+                       const int32_t *root_token_host, const int32_t *base_pos_host, int32_t B, float delta,
+                       const opt_tree_host_out *out, void *stream);
+
+/* Reads (and clears) the device status word; synchronises the device.  *status_host is
+ * OPT_TREE_OK or the first device-side error recorded since the last call. */
+int opt_tree_last_device_status(opt_tree_ctx *ctx, int32_t *status_host);
+
+/* Number of kernels the library has launched through this context since it was created. */
+int64_t opt_tree_launch_count(const opt_tree_ctx *ctx);
+
+const char *opt_tree_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OPT_TREE_H_ */

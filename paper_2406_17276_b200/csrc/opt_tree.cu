@@ -1,0 +1,532 @@
+// OPT-Tree draft-tree construction, tree mask and greedy verification for B200 (sm_100a):
+// kernels and the C ABI declared in include/opt_tree.h.
+#include "../../include/opt_tree.h"
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <new>
+#include <stdio.h>
+#include <string.h>
+
+#include "select.cuh"
+
+namespace ot {
+
+constexpr int kRowMul = 31;                 // row of (token t, depth d) = (t*31 + d) mod H
+
+__device__ __forceinline__ int row_of(int token, int depth, int H) {
+    return (int)(((long long)token * kRowMul + depth) % H);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Workspace
+// ------------------------------------------------------------------------------------------------
+struct Workspace {
+    // build
+    double* cand_phat;     // [B][n*k]
+    int32_t* cand_tok;     // [B][n*k]
+    int32_t* T_tok;        // [B][D*n]
+    int32_t* T_par;        // [B][D*n]
+    double* T_phat;        // [B][D*n]
+    int32_t* R;            // [B][2][n]
+    double* E_prev;        // [B]
+    int32_t* st;           // [B][8]
+    // verify
+    int32_t* g;            // [B][n+1]  target argmax after the root (0) and after node i (i+1)
+    int32_t* vdone;        // [B]
+    int32_t* status;       // [1]
+    // device copies of inputs / outputs for the host-buffer step
+    int32_t *h_root, *h_base;                          // [B]
+    int32_t *o_token, *o_parent, *o_depth; double* o_phat;
+    int32_t *o_nsel, *o_dreach; double* o_elen;
+    uint64_t* o_mask; int32_t* o_pos;
+    int32_t *o_alen, *o_atok, *o_anode, *o_next;
+};
+
+struct Layout {
+    size_t total = 0;
+    template <class T> size_t take(size_t count) {
+        size_t off = (total + 255) & ~(size_t)255;
+        total = off + count * sizeof(T);
+        return off;
+    }
+};
+
+static size_t carve(const opt_tree_config& c, char* base, Workspace* w) {
+    const size_t B = c.max_batch, n = c.n, k = c.k, D = c.max_depth, W = (c.n + 63) / 64;
+    Layout L;
+    size_t o;
+#define OT_TAKE(field, T, count) o = L.take<T>(count); if (w) w->field = reinterpret_cast<T*>(base + o);
+    OT_TAKE(cand_phat, double, B * n * k)
+    OT_TAKE(cand_tok, int32_t, B * n * k)
+    OT_TAKE(T_tok, int32_t, B * D * n)
+    OT_TAKE(T_par, int32_t, B * D * n)
+    OT_TAKE(T_phat, double, B * D * n)
+    OT_TAKE(R, int32_t, B * 2 * n)
+    OT_TAKE(E_prev, double, B)
+    OT_TAKE(st, int32_t, B * 8)
+    OT_TAKE(g, int32_t, B * (n + 1))
+    OT_TAKE(vdone, int32_t, B)
+    OT_TAKE(status, int32_t, 1)
+    OT_TAKE(h_root, int32_t, B)
+    OT_TAKE(h_base, int32_t, B)
+    OT_TAKE(o_token, int32_t, B * n)
+    OT_TAKE(o_parent, int32_t, B * n)
+    OT_TAKE(o_depth, int32_t, B * n)
+    OT_TAKE(o_phat, double, B * n)
+    OT_TAKE(o_nsel, int32_t, B)
+    OT_TAKE(o_dreach, int32_t, B)
+    OT_TAKE(o_elen, double, B)
+    OT_TAKE(o_mask, uint64_t, B * n * W)
+    OT_TAKE(o_pos, int32_t, B * n)
+    OT_TAKE(o_alen, int32_t, B)
+    OT_TAKE(o_atok, int32_t, B * (D + 1))
+    OT_TAKE(o_anode, int32_t, B * D)
+    OT_TAKE(o_next, int32_t, B)
+#undef OT_TAKE
+    return (L.total + 255) & ~(size_t)255;
+}
+
+struct Params {            // by-value kernel parameters common to the build kernels
+    int V, H, n, k, kk, Dcap, max_depth;
+    float delta;
+    int aligned;
+};
+
+__device__ __forceinline__ SeqWork seq_work(const Workspace& w, const Params& p, int b) {
+    SeqWork s;
+    s.cand_phat = w.cand_phat + (size_t)b * p.n * p.k;
+    s.cand_tok = w.cand_tok + (size_t)b * p.n * p.k;
+    s.T_tok = w.T_tok + (size_t)b * p.max_depth * p.n;
+    s.T_par = w.T_par + (size_t)b * p.max_depth * p.n;
+    s.T_phat = w.T_phat + (size_t)b * p.max_depth * p.n;
+    s.R = w.R + (size_t)b * 2 * p.n;
+    s.E_prev = w.E_prev + b;
+    s.st = w.st + (size_t)b * 8;
+    return s;
+}
+__device__ __forceinline__ TreeOut tree_out(const opt_tree_out& o, const Params& p, int b) {
+    TreeOut t;
+    t.token = o.token + (size_t)b * p.n;
+    t.parent = o.parent + (size_t)b * p.n;
+    t.depth = o.depth + (size_t)b * p.n;
+    t.phat = o.phat + (size_t)b * p.n;
+    t.n_sel = o.n_sel + b;
+    t.depth_reached = o.depth_reached + b;
+    t.expected_len = o.expected_len + b;
+    t.esub_trace = o.esub_trace ? o.esub_trace + (size_t)b * p.max_depth : nullptr;
+    return t;
+}
+
+__device__ __forceinline__ void init_barriers(BlockSmem& s) {
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) mbar_init(&s.full_bar[i], 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Kernels
+// ------------------------------------------------------------------------------------------------
+__global__ void init_build_kernel(Workspace w, int B) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int32_t* st = w.st + (size_t)b * 8;
+    st[kStFsize] = 1; st[kStActive] = 1; st[kStDone] = 0; st[kStNR] = 0; st[kStDepth] = 0;
+    w.E_prev[b] = 0.0;
+}
+
+// One drafting step (layer d) of Algorithm 1: CTA (slot, b) expands frontier node `slot` of
+// sequence b; the CTA that finishes a sequence's last row also selects the layer.
+__global__ void __launch_bounds__(kThreads)
+build_round_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, const int32_t* __restrict__ root_token,
+                   opt_tree_out out, int d) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    BlockSmem& s = *reinterpret_cast<BlockSmem*>(smem_raw);
+    const int b = blockIdx.y, slot = blockIdx.x, tid = threadIdx.x;
+    const SeqWork sw = seq_work(w, p, b);
+    if (!__ldcg(&sw.st[kStActive])) return;
+    const int fsize = __ldcg(&sw.st[kStFsize]);
+    if (slot >= fsize) return;
+    init_barriers(s);
+
+    int token, depth;
+    double parent_phat;
+    if (d == 1) {
+        token = root_token[b]; depth = 0; parent_phat = 1.0;       // the root counts as factor 1 (Eq. 2)
+    } else {
+        const int gid = (d - 2) * p.n + slot;
+        token = __ldcg(&sw.T_tok[gid]); depth = d - 1; parent_phat = __ldcg(&sw.T_phat[gid]);
+    }
+    if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
+    const uint16_t* row = draft + (size_t)row_of(token, depth, p.H) * p.V;
+
+    uint32_t parity = 0;
+    RowResult res;
+    const bool ok = row_softmax_topk(s, row, p.V, p.k, p.aligned != 0, parity, w.status, res);
+    if (tid < p.k) {
+        double ph = -1.0; int32_t tk = -1;
+        if (ok && tid < res.kk) {
+            const unsigned long long key = s.win[tid];
+            tk = (int32_t)cand_token(key);
+            ph = parent_phat * (exp((double)cand_logit(key) - res.m) / res.S);   // Eq. 2
+        }
+        sw.cand_phat[slot * p.k + tid] = ph;
+        sw.cand_tok[slot * p.k + tid] = tk;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s.flag = (atomicAdd(&sw.st[kStDone], 1) == fsize - 1);
+    __syncthreads();
+    if (!s.flag) return;
+    __threadfence();
+    finish_layer(s, sw, tree_out(out, p, b), d, p.n, p.k, p.kk, p.Dcap, p.max_depth, p.delta);
+}
+
+// The row step alone, one CTA per listed row.
+__global__ void __launch_bounds__(kThreads)
+row_topk_kernel(Params p, const uint16_t* __restrict__ logits, const int32_t* __restrict__ rows,
+                int32_t* tok_out, double* prob_out, int* status) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    BlockSmem& s = *reinterpret_cast<BlockSmem*>(smem_raw);
+    init_barriers(s);
+    int r = rows[blockIdx.x];
+    if (r < 0 || r >= p.H) { set_status(status, kErrInternal); r = 0; }
+    uint32_t parity = 0;
+    RowResult res;
+    const bool ok = row_softmax_topk(s, logits + (size_t)r * p.V, p.V, p.k, p.aligned != 0, parity, status, res);
+    const int tid = threadIdx.x;
+    if (tid < p.k) {
+        double pr = 0.0; int32_t tk = -1;
+        if (ok && tid < res.kk) {
+            const unsigned long long key = s.win[tid];
+            tk = (int32_t)cand_token(key);
+            pr = exp((double)cand_logit(key) - res.m) / res.S;
+        }
+        tok_out[(size_t)blockIdx.x * p.k + tid] = tk;
+        prob_out[(size_t)blockIdx.x * p.k + tid] = pr;
+    }
+}
+
+// Tree attention mask + position ids: one CTA per sequence, one thread per node.
+__global__ void __launch_bounds__(kThreads)
+mask_kernel(const int32_t* __restrict__ parent, const int32_t* __restrict__ depth, const int32_t* __restrict__ n_sel,
+            const int32_t* __restrict__ base_pos, int n, uint64_t* mask, int32_t* position_ids, int* status) {
+    const int b = blockIdx.x, i = threadIdx.x;
+    if (i >= n) return;
+    const int W = (n + 63) >> 6;
+    const int ns = n_sel[b];
+    const int32_t* par = parent + (size_t)b * n;
+    uint64_t bits[kMaxN / 64] = {0, 0, 0, 0};
+    int pos = 0;
+    if (i < ns) {
+        int a = i, steps = 0;
+        while (a >= 0 && steps <= n) {                      // an ancestor chain is at most n long
+            if (a >= n) { set_status(status, kErrInternal); break; }
+#pragma unroll
+            for (int wd = 0; wd < kMaxN / 64; ++wd)
+                if ((a >> 6) == wd) bits[wd] |= 1ull << (a & 63);
+            a = par[a];
+            ++steps;
+        }
+        pos = (base_pos ? base_pos[b] : 0) + depth[(size_t)b * n + i];
+    }
+#pragma unroll
+    for (int wd = 0; wd < kMaxN / 64; ++wd)
+        if (wd < W) mask[((size_t)b * n + i) * W + wd] = bits[wd];
+    position_ids[(size_t)b * n + i] = pos;
+}
+
+__device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+struct VerifySmem {
+    unsigned long long red_u64[kWarps];
+    int flag;
+    int hit;
+};
+
+// Greedy verification.  CTA (j, b): j = 0 takes the target row after the root, j >= 1 the row after
+// kept node j-1; each finds the row's argmax (lowest token on ties).  The last CTA of a sequence
+// then walks the tree: accept the child that carries the target's token, until none does.
+__global__ void __launch_bounds__(kThreads)
+verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const int32_t* __restrict__ root_token,
+              opt_tree_out tree, int32_t* accept_len, int32_t* accept_tokens, int32_t* accept_nodes, int32_t* next_root) {
+    __shared__ VerifySmem s;
+    const int b = blockIdx.y, j = blockIdx.x, tid = threadIdx.x;
+    const int ns = tree.n_sel[b];
+    if (j > ns) return;
+    const int32_t* tok = tree.token + (size_t)b * p.n;
+    const int32_t* par = tree.parent + (size_t)b * p.n;
+    int token = j == 0 ? root_token[b] : tok[j - 1];
+    const int depth = j == 0 ? 0 : tree.depth[(size_t)b * p.n + j - 1];
+    if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
+    const uint16_t* row = target + (size_t)row_of(token, depth, p.H) * p.V;
+
+    unsigned long long best_key = 0ull;
+    if (p.aligned) {
+        const uint4* vec = reinterpret_cast<const uint4*>(row);
+        const int nv = p.V >> 3;
+        float best = -INFINITY;
+        int best_v = -1;
+        int v = tid;
+        for (; v + 3 * kThreads < nv; v += 4 * kThreads) {
+            uint4 q[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) q[u] = ld_nc_v4(vec + v + u * kThreads);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t m2 = max_bf16x2(max_bf16x2(q[u].x, q[u].y), max_bf16x2(q[u].z, q[u].w));
+                const float f = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
+                if (f > best || best_v < 0) { best = f; best_v = v + u * kThreads; }
+            }
+        }
+        for (; v < nv; v += kThreads) {
+            const uint4 q = ld_nc_v4(vec + v);
+            const uint32_t m2 = max_bf16x2(max_bf16x2(q.x, q.y), max_bf16x2(q.z, q.w));
+            const float f = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
+            if (f > best || best_v < 0) { best = f; best_v = v; }
+        }
+        if (best_v >= 0) {
+            const uint4 q = vec[best_v];
+            const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int e = 7; e >= 0; --e) {
+                const uint32_t bits = (e & 1) ? (ww[e >> 1] >> 16) : (ww[e >> 1] & 0xFFFFu);
+                if (bf16_bits_to_float(bits) == best) best_key = cand_key(bits, (uint32_t)(best_v * 8 + e));
+            }
+        }
+    } else {
+        for (int v = tid; v < p.V; v += kThreads) {
+            const unsigned long long key = cand_key(__ldg(row + v), (uint32_t)v);
+            best_key = key > best_key ? key : best_key;
+        }
+    }
+    best_key = block_max_u64(best_key, s.red_u64);
+    int32_t* g = w.g + (size_t)b * (p.n + 1);
+    if (tid == 0) g[j] = (int32_t)cand_token(best_key);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s.flag = (atomicAdd(&w.vdone[b], 1) == ns);
+    __syncthreads();
+    if (!s.flag) return;
+    __threadfence();
+
+    // acceptance walk (block-wide child search; children of one node carry distinct tokens)
+    int32_t* at = accept_tokens + (size_t)b * (p.max_depth + 1);
+    int32_t* an = accept_nodes + (size_t)b * p.max_depth;
+    for (int i = tid; i <= p.max_depth; i += kThreads) at[i] = -1;
+    for (int i = tid; i < p.max_depth; i += kThreads) an[i] = -1;
+    __syncthreads();
+    int cur = -1, A = 0;
+    for (int step = 0; step <= p.max_depth; ++step) {
+        const int y = __ldcg(&g[cur + 1]);
+        if (tid == 0) { at[A] = y; s.hit = -1; }
+        ++A;
+        __syncthreads();
+        if (A > p.max_depth) break;
+        for (int i = tid; i < ns; i += kThreads)
+            if (par[i] == cur && tok[i] == y) s.hit = i;
+        __syncthreads();
+        const int hit = s.hit;
+        __syncthreads();
+        if (hit < 0) break;
+        if (tid == 0) an[A - 1] = hit;
+        cur = hit;
+    }
+    if (tid == 0) {
+        accept_len[b] = A;
+        next_root[b] = __ldcg(&g[cur + 1]);
+        w.vdone[b] = 0;
+    }
+}
+
+}  // namespace ot
+
+// ------------------------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------------------------
+struct opt_tree_ctx {
+    opt_tree_config cfg;
+    ot::Workspace ws;
+    void* base;
+    size_t bytes;
+    int device;
+    int64_t launches;
+};
+
+namespace {
+
+bool valid_cfg(const opt_tree_config* c) {
+    return c && c->V >= 1 && c->H >= 1 && c->n >= 1 && c->k >= 1 && c->max_depth >= 1 && c->max_batch >= 1;
+}
+int supported_cfg(const opt_tree_config* c) {
+    if (c->n > OPT_TREE_MAX_N || c->k > OPT_TREE_MAX_K || c->k > c->V) return OPT_TREE_ERR_UNSUPPORTED;
+    if ((long long)c->V * 31 + c->max_depth > 2147483647LL) return OPT_TREE_ERR_UNSUPPORTED;
+    return OPT_TREE_OK;
+}
+ot::Params make_params(const opt_tree_ctx* ctx, const void* table, float delta) {
+    const opt_tree_config& c = ctx->cfg;
+    ot::Params p;
+    p.V = c.V; p.H = c.H; p.n = c.n; p.k = c.k; p.kk = c.k < c.V ? c.k : c.V;
+    p.Dcap = c.max_depth < c.n ? c.max_depth : c.n;
+    p.max_depth = c.max_depth;
+    p.delta = delta;
+    p.aligned = ((reinterpret_cast<uintptr_t>(table) & 15u) == 0 && (c.V % 8) == 0) ? 1 : 0;
+    return p;
+}
+bool bad_tree(const opt_tree_out* t) {
+    return !t || !t->token || !t->parent || !t->depth || !t->phat || !t->n_sel || !t->depth_reached || !t->expected_len;
+}
+int check_launch() { return cudaGetLastError() == cudaSuccess ? OPT_TREE_OK : OPT_TREE_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+size_t opt_tree_workspace_bytes(const opt_tree_config* cfg) {
+    if (!valid_cfg(cfg) || supported_cfg(cfg) != OPT_TREE_OK) return 0;
+    return ot::carve(*cfg, nullptr, nullptr);
+}
+
+int opt_tree_create(opt_tree_ctx** out, const opt_tree_config* cfg) {
+    if (!out) return OPT_TREE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!valid_cfg(cfg)) return OPT_TREE_ERR_INVALID_ARG;
+    int rc = supported_cfg(cfg);
+    if (rc != OPT_TREE_OK) return rc;
+    opt_tree_ctx* ctx = new (std::nothrow) opt_tree_ctx();
+    if (!ctx) return OPT_TREE_ERR_CUDA;
+    ctx->cfg = *cfg;
+    ctx->launches = 0;
+    ctx->bytes = ot::carve(*cfg, nullptr, nullptr);
+    if (cudaGetDevice(&ctx->device) != cudaSuccess || cudaMalloc(&ctx->base, ctx->bytes) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx;
+        return OPT_TREE_ERR_CUDA;
+    }
+    ot::carve(*cfg, static_cast<char*>(ctx->base), &ctx->ws);
+    bool ok = cudaMemset(ctx->base, 0, ctx->bytes) == cudaSuccess;
+    ok = ok && cudaFuncSetAttribute(ot::build_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)sizeof(ot::BlockSmem)) == cudaSuccess;
+    ok = ok && cudaFuncSetAttribute(ot::row_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)sizeof(ot::BlockSmem)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        cudaFree(ctx->base);
+        delete ctx;
+        return OPT_TREE_ERR_CUDA;
+    }
+    *out = ctx;
+    return OPT_TREE_OK;
+}
+
+int opt_tree_destroy(opt_tree_ctx* ctx) {
+    if (!ctx) return OPT_TREE_ERR_INVALID_ARG;
+    cudaError_t e = cudaFree(ctx->base);
+    delete ctx;
+    return e == cudaSuccess ? OPT_TREE_OK : OPT_TREE_ERR_CUDA;
+}
+
+int opt_tree_build(opt_tree_ctx* ctx, const void* draft, const int32_t* root_token, int32_t B, float delta,
+                   const opt_tree_out* out, void* stream) {
+    if (!ctx || !draft || !root_token || bad_tree(out) || B < 1 || delta != delta) return OPT_TREE_ERR_INVALID_ARG;
+    if (B > ctx->cfg.max_batch) return OPT_TREE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const ot::Params p = make_params(ctx, draft, delta);
+    ot::init_build_kernel<<<(B + 255) / 256, 256, 0, st>>>(ctx->ws, B);
+    ctx->launches++;
+    for (int d = 1; d <= p.Dcap; ++d) {
+        const int width = d == 1 ? 1 : (d == 2 ? (p.kk < p.n ? p.kk : p.n) : p.n);   // largest possible frontier
+        ot::build_round_kernel<<<dim3(width, B), ot::kThreads, sizeof(ot::BlockSmem), st>>>(
+            ctx->ws, p, static_cast<const uint16_t*>(draft), root_token, *out, d);
+        ctx->launches++;
+    }
+    return check_launch();
+}
+
+int opt_tree_mask(opt_tree_ctx* ctx, const opt_tree_out* tree, int32_t B, const int32_t* base_pos, uint64_t* mask,
+                  int32_t* position_ids, void* stream) {
+    if (!ctx || bad_tree(tree) || !mask || !position_ids || B < 1 || B > ctx->cfg.max_batch) return OPT_TREE_ERR_INVALID_ARG;
+    ot::mask_kernel<<<B, ot::kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        tree->parent, tree->depth, tree->n_sel, base_pos, ctx->cfg.n, mask, position_ids, ctx->ws.status);
+    ctx->launches++;
+    return check_launch();
+}
+
+int opt_tree_verify(opt_tree_ctx* ctx, const opt_tree_out* tree, const void* target, const int32_t* root_token, int32_t B,
+                    int32_t* accept_len, int32_t* accept_tokens, int32_t* accept_nodes, int32_t* next_root, void* stream) {
+    if (!ctx || bad_tree(tree) || !target || !root_token || !accept_len || !accept_tokens || !accept_nodes || !next_root ||
+        B < 1 || B > ctx->cfg.max_batch)
+        return OPT_TREE_ERR_INVALID_ARG;
+    const ot::Params p = make_params(ctx, target, 0.0f);
+    ot::verify_kernel<<<dim3(ctx->cfg.n + 1, B), ot::kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        ctx->ws, p, static_cast<const uint16_t*>(target), root_token, *tree, accept_len, accept_tokens, accept_nodes, next_root);
+    ctx->launches++;
+    return check_launch();
+}
+
+int opt_tree_row_softmax_topk(opt_tree_ctx* ctx, const void* logits, const int32_t* rows, int32_t nrows, int32_t* tok_out,
+                              double* prob_out, void* stream) {
+    if (!ctx || !logits || !rows || !tok_out || !prob_out || nrows < 0) return OPT_TREE_ERR_INVALID_ARG;
+    if (nrows == 0) return OPT_TREE_OK;
+    const ot::Params p = make_params(ctx, logits, 0.0f);
+    ot::row_topk_kernel<<<nrows, ot::kThreads, sizeof(ot::BlockSmem), static_cast<cudaStream_t>(stream)>>>(
+        p, static_cast<const uint16_t*>(logits), rows, tok_out, prob_out, ctx->ws.status);
+    ctx->launches++;
+    return check_launch();
+}
+
+int opt_tree_step_host(opt_tree_ctx* ctx, const void* draft, const void* target, const int32_t* root_host,
+                       const int32_t* base_host, int32_t B, float delta, const opt_tree_host_out* ho, void* stream) {
+    if (!ctx || !draft || !target || !root_host || !ho || B < 1 || B > ctx->cfg.max_batch) return OPT_TREE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const ot::Workspace& w = ctx->ws;
+    const size_t n = ctx->cfg.n, D = ctx->cfg.max_depth, W = (ctx->cfg.n + 63) / 64, Bz = B;
+    bool ok = cudaMemcpyAsync(w.h_root, root_host, Bz * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (base_host) ok = ok && cudaMemcpyAsync(w.h_base, base_host, Bz * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) return OPT_TREE_ERR_CUDA;
+    opt_tree_out t = {w.o_token, w.o_parent, w.o_depth, w.o_phat, w.o_nsel, w.o_dreach, w.o_elen, nullptr};
+    int rc = opt_tree_build(ctx, draft, w.h_root, B, delta, &t, stream);
+    if (rc == OPT_TREE_OK) rc = opt_tree_mask(ctx, &t, B, base_host ? w.h_base : nullptr, w.o_mask, w.o_pos, stream);
+    if (rc == OPT_TREE_OK) rc = opt_tree_verify(ctx, &t, target, w.h_root, B, w.o_alen, w.o_atok, w.o_anode, w.o_next, stream);
+    if (rc != OPT_TREE_OK) return rc;
+#define OT_D2H(dst, src, bytes) if (ok && (dst)) ok = cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    OT_D2H(ho->token, w.o_token, Bz * n * 4) OT_D2H(ho->parent, w.o_parent, Bz * n * 4) OT_D2H(ho->depth, w.o_depth, Bz * n * 4)
+    OT_D2H(ho->phat, w.o_phat, Bz * n * 8) OT_D2H(ho->n_sel, w.o_nsel, Bz * 4) OT_D2H(ho->depth_reached, w.o_dreach, Bz * 4)
+    OT_D2H(ho->expected_len, w.o_elen, Bz * 8) OT_D2H(ho->mask, w.o_mask, Bz * n * W * 8) OT_D2H(ho->position_ids, w.o_pos, Bz * n * 4)
+    OT_D2H(ho->accept_len, w.o_alen, Bz * 4) OT_D2H(ho->accept_tokens, w.o_atok, Bz * (D + 1) * 4)
+    OT_D2H(ho->accept_nodes, w.o_anode, Bz * D * 4) OT_D2H(ho->next_root, w.o_next, Bz * 4)
+#undef OT_D2H
+    if (!ok || cudaStreamSynchronize(st) != cudaSuccess) return OPT_TREE_ERR_CUDA;
+    return OPT_TREE_OK;
+}
+
+int opt_tree_last_device_status(opt_tree_ctx* ctx, int32_t* status_host) {
+    if (!ctx || !status_host) return OPT_TREE_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return OPT_TREE_ERR_CUDA;
+    if (cudaMemcpy(status_host, ctx->ws.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return OPT_TREE_ERR_CUDA;
+    if (cudaMemset(ctx->ws.status, 0, 4) != cudaSuccess) return OPT_TREE_ERR_CUDA;
+    return OPT_TREE_OK;
+}
+
+int64_t opt_tree_launch_count(const opt_tree_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* opt_tree_strerror(int code) {
+    switch (code) {
+        case OPT_TREE_OK: return "ok";
+        case OPT_TREE_ERR_INVALID_ARG: return "invalid argument";
+        case OPT_TREE_ERR_UNSUPPORTED: return "unsupported configuration";
+        case OPT_TREE_ERR_CUDA: return "CUDA runtime error";
+        case OPT_TREE_ERR_TIMEOUT: return "device-side wait timed out";
+        case OPT_TREE_ERR_INTERNAL: return "device-side bounds check failed";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

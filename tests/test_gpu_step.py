@@ -1,0 +1,120 @@
+"""-m gpu: whole decoding steps (build, mask, verify) through the C ABI against the oracle."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2406_17276_b200 import binding, synth
+from tests import _compare
+from tests._gpu import dev_table, gpu_step
+
+pytestmark = pytest.mark.gpu
+NEG_INF = -math.inf
+
+
+def _run(w, deltas, steps=1, H=None, V=None, chain=False):
+    ld, lt = synth.make_tables(w, H=H, V=V)
+    Hh, Vv = ld.shape
+    ot = binding.OptTree(Vv, Hh, w.n, w.k, w.max_depth, w.batch)
+    d_ld, d_lt = dev_table(ld), dev_table(lt)
+    memo = oracle.Memo(w.k, cap=4 * Hh)
+    total = dict(exact=0, near_tie=0, stop_near_tie=0, max_phat_rel=0.0, max_elen_rel=0.0)
+    for delta in deltas:
+        roots = synth.root_tokens(w.batch, Vv, w.seed + 1)
+        base = np.arange(w.batch, dtype=np.int32) * 7 + 3
+        for _ in range(steps):
+            g = gpu_step(ot, d_ld, d_lt, roots, delta, base)
+            o, st = _compare.compare_step(w, ld, lt, roots, delta, g, base_pos=base, memo=memo)
+            for k2 in ("exact", "near_tie", "stop_near_tie"):
+                total[k2] += st[k2]
+            for k2 in ("max_phat_rel", "max_elen_rel"):
+                total[k2] = max(total[k2], st[k2])
+            roots = o.next_root.copy()           # the oracle's token feeds the next step (Algorithm 2, Concat)
+            base = base + o.accept_len
+    return total
+
+
+@pytest.mark.parametrize("name,V,H", [("c1", 20000, 512), ("c2", 20000, 512), ("c4", 20000, 512), ("c4", 8200, 256),
+                                      ("c3", 40008, 128), ("c5", 40008, 128)])
+def test_reduced_tables_all_thresholds(name, V, H):
+    w = synth.WORKLOADS[name]
+    t = _run(w, [NEG_INF, 0.0, 0.2, 0.7], steps=3, H=H, V=V)
+    assert t["exact"] > 0 and t["near_tie"] + t["stop_near_tie"] <= 0.05 * (t["exact"] + 1)
+    print(name, V, t)
+
+
+@pytest.mark.parametrize("name,steps", [("c1", 20), ("c2", 10), ("c3", 3), ("c4", 3), ("c5", 1)])
+def test_full_size_configurations(name, steps):
+    w = synth.WORKLOADS[name]
+    t = _run(w, [NEG_INF] if name == "c5" else [NEG_INF, 0.2], steps=steps)
+    assert t["exact"] > 0 and t["near_tie"] + t["stop_near_tie"] <= 0.05 * (t["exact"] + 1)
+    print(name, t)
+
+
+@pytest.mark.parametrize("n,k,D,B,V", [(1, 4, 5, 3, 512), (6, 1, 6, 3, 512), (256, 32, 20, 2, 4096), (5, 8, 3, 4, 8),
+                                       (7, 3, 4, 2, 12), (64, 10, 10, 1, 32000), (10, 10, 6, 5, 100)])
+def test_degenerate_and_maximum_sizes(n, k, D, B, V):
+    w = synth.Workload("edge", B, V, n, k, D, 3.0, 1.1, 0.3, H=64, seed=n * 1000 + k)
+    t = _run(w, [NEG_INF, 0.1], steps=2)
+    assert t["exact"] > 0
+    print(t)
+
+
+def test_two_runs_are_bit_identical():
+    w = synth.WORKLOADS["c4"]
+    ld, lt = synth.make_tables(w, H=256, V=20000)
+    ot = binding.OptTree(20000, 256, w.n, w.k, w.max_depth, w.batch)
+    d_ld, d_lt = dev_table(ld), dev_table(lt)
+    roots = synth.root_tokens(w.batch, 20000, 9)
+    a = gpu_step(ot, d_ld, d_lt, roots, 0.2)
+    b = gpu_step(ot, d_ld, d_lt, roots, 0.2)
+    for f in a:
+        assert np.array_equal(a[f], b[f], equal_nan=True), f
+
+
+def test_identical_tables_accept_at_least_two_tokens():
+    w = synth.Workload("same", 8, 8200, 24, 6, 8, 3.0, 1.1, 0.0, H=128, seed=77)
+    ld, _ = synth.make_tables(w)
+    ot = binding.OptTree(w.V, w.H, w.n, w.k, w.max_depth, w.batch)
+    d = dev_table(ld)
+    g = gpu_step(ot, d, d, synth.root_tokens(8, w.V, 1), NEG_INF)
+    assert np.all(g["accept_len"] >= 2)
+
+
+def test_host_buffer_step_matches_device_path():
+    w = synth.WORKLOADS["c4"]
+    ld, lt = synth.make_tables(w, H=256, V=20000)
+    ot = binding.OptTree(20000, 256, w.n, w.k, w.max_depth, w.batch)
+    d_ld, d_lt = dev_table(ld), dev_table(lt)
+    roots = synth.root_tokens(w.batch, 20000, 4)
+    base = np.arange(w.batch, dtype=np.int32)
+    g = gpu_step(ot, d_ld, d_lt, roots, 0.2, base)
+    ho = ot.alloc_host_out(w.batch)
+    ot.step_host(d_ld, d_lt, torch.from_numpy(roots).pin_memory(), torch.from_numpy(base).pin_memory(), 0.2, ho)
+    for f, t in ho.items():
+        assert np.array_equal(t.numpy(), g[f]), f
+
+
+def test_argument_checks_return_status_codes():
+    with pytest.raises(binding.OptTreeError) as e:
+        binding.OptTree(32000, 64, 257, 10, 10, 1)
+    assert e.value.code == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.OptTreeError) as e:
+        binding.OptTree(32000, 64, 64, 33, 10, 1)
+    assert e.value.code == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.OptTreeError) as e:
+        binding.OptTree(8, 64, 4, 9, 3, 1)                   # k > V
+    assert e.value.code == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.OptTreeError) as e:
+        binding.OptTree(0, 64, 4, 2, 3, 1)
+    assert e.value.code == binding.ERR_INVALID_ARG
+    ot = binding.OptTree(512, 64, 8, 4, 4, 2)
+    tab = torch.zeros((64, 512), dtype=torch.int16, device="cuda")
+    with pytest.raises(binding.OptTreeError) as e:
+        ot.build(tab, torch.zeros(3, dtype=torch.int32, device="cuda"), 0.0)     # B > max_batch
+    assert e.value.code == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.OptTreeError) as e:
+        ot.build(tab, torch.zeros(2, dtype=torch.int32, device="cuda"), float("nan"))
+    assert e.value.code == binding.ERR_INVALID_ARG
