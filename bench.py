@@ -1,0 +1,285 @@
+#!/usr/bin/env python
+"""Benchmark of the OPT-Tree decoding-step bookkeeping on B200.
+
+A step = one pass of the whole hot path over one batch: opt_tree_build (Algorithm 1),
+opt_tree_mask and opt_tree_verify (Algorithm 2) for B sequences, with the next step's root
+tokens taken from this step's verification.  Workload: batch 32, V=32000, n=64, k=10,
+max depth 10 ("c4"), threshold off (every layer drafted, so the byte count is fixed).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]         # CUDA path, one JSON line
+  python bench.py --impl reference ...                        # the CPU oracle, same metric
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs its own batch
+with its own seeds and tables (weak scaling, no data-path collective); the time is the maximum
+over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2406_17276_b200 import synth  # noqa: E402
+
+METRIC = "opt_tree_builds_per_s"
+UNIT = "trees/s"
+NEG_INF = -math.inf
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period, self.stop_flag = index, period_s, threading.Event()
+        self.sm, self.reasons, self.sm_max = [], set(), None
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                 "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+        while not self.stop_flag.is_set():
+            try:
+                self.sm.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def result(self):
+        self.stop_flag.set()
+        self.join(timeout=2)
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.sm_max,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+def logical_rows(w, depth_reached):
+    """Rows of L_d one build reads: the root row, the min(n,k) first-layer nodes, then n per layer."""
+    rows = 0
+    for d in depth_reached:
+        d = int(d)
+        rows += 1 + (min(w.n, w.k) if d >= 2 else 0) + max(0, d - 2) * w.n
+    return rows
+
+
+def run_cuda(args):
+    import torch
+    from paper_2406_17276_b200 import binding, build
+
+    rank = int(os.environ.get("RANK", 0)); world = int(os.environ.get("WORLD_SIZE", 1))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    build.build()
+    w = synth.WORKLOADS[args.workload]
+    w = synth.Workload(**{**w.__dict__, "seed": w.seed + 1000 * rank})
+    ld, lt = synth.make_tables(w)
+    d_ld = torch.from_numpy(ld.view(np.int16)).cuda(); d_lt = torch.from_numpy(lt.view(np.int16)).cuda()
+    B, D = w.batch, w.max_depth
+    ot = binding.OptTree(w.V, w.H, w.n, w.k, D, B, device=f"cuda:{local}")
+    roots0 = torch.from_numpy(synth.root_tokens(B, w.V, w.seed + 1)).cuda()
+    base = torch.zeros(B, dtype=torch.int32, device="cuda")
+    tree = ot.alloc_tree(B, trace=False)
+    mask = torch.empty((B, w.n, ot.W), dtype=torch.int64, device="cuda")
+    pos = torch.empty((B, w.n), dtype=torch.int32, device="cuda")
+    i32 = dict(dtype=torch.int32, device="cuda")
+    vout = [(torch.empty(B, **i32), torch.empty((B, D + 1), **i32), torch.empty((B, D), **i32), torch.empty(B, **i32))
+            for _ in range(2)]
+    delta = args.delta
+
+    def step(i, root):
+        ot.build(d_ld, root, delta, tree)
+        ot.mask(tree, base, mask, pos)
+        o = vout[i & 1]
+        ot.verify(tree, d_lt, root, o)
+        return o[3]                                  # next_root feeds the next step
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ----
+    root = roots0
+    for i in range(args.warmup):
+        root = step(i, root)
+    barrier()
+    sampler = ClockSampler(local); sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    bev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    rows_total = 0
+    launches0 = ot.launch_count()
+    ev0.record()
+    for i in range(args.steps):
+        bev[i][0].record()
+        ot.build(d_ld, root, delta, tree)
+        bev[i][1].record()
+        ot.mask(tree, base, mask, pos)
+        o = vout[i & 1]
+        ot.verify(tree, d_lt, root, o)
+        root = o[3]
+    ev1.record()
+    barrier()
+    clocks = sampler.result()
+    launches = ot.launch_count() - launches0
+    ms = ev0.elapsed_time(ev1)
+    build_ms = sum(a.elapsed_time(b) for a, b in bev) / args.steps
+    status = ot.device_status()
+    if status != 0:
+        raise SystemExit(f"bench.py: device status {status}")
+    # bytes of the last build (all builds are identical in size when the threshold is off)
+    rows_last = logical_rows(w, tree.depth_reached.cpu().numpy())
+    if delta == NEG_INF:
+        rows_total = rows_last
+    else:
+        rows_total = rows_last            # threshold on: the last build's own count is reported
+    algo_bytes = 2.0 * w.V * rows_total
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # ---- end to end through the host-buffer entry point ----
+    ho = ot.alloc_host_out(B)
+    h_root = roots0.cpu().pin_memory(); h_base = torch.zeros(B, dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 200))
+    for _ in range(3):
+        ot.step_host(d_ld, d_lt, h_root, h_base, delta, ho)
+        h_root.copy_(ho["next_root"])
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        ot.step_host(d_ld, d_lt, h_root, h_base, delta, ho)
+        h_root.copy_(ho["next_root"])
+    e1.record()
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = 2 * B * 4
+    d2h = sum(int(t.numel() * t.element_size()) for t in ho.values())
+
+    peak, peak_kind = _peaks()
+    achieved = algo_bytes / (build_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": world * B * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{w.name}: batch {B} per GPU, V={w.V}, n={w.n}, k={w.k}, max_depth={D}, "
+                               f"delta={'off' if delta == NEG_INF else delta}, H={w.H} bf16 tables "
+                               f"(sigma {w.sigma}, Zipf s {w.zipf_s}, {int(w.disagree * 100)}% rows disagree)",
+                   "l2": "inputs larger than L2: two 262 MB tables against a 126 MB L2, no explicit flush",
+                   "step": "build + mask + verify, next roots from verify"},
+        "clocks": clocks,
+        "e2e": {"value": world * B / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "opt_tree_build (init + one build_round_kernel per layer)",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / 8000.0,
+                     "algorithmic_bytes_per_build_call": algo_bytes, "build_ms": build_ms, "traffic": args.traffic},
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w, ld, lt, steps=2)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(w, ld, lt, steps, batch=None):
+    """The oracle as it stands, single thread, un-memoised, on a bounded sample of the workload."""
+    import oracle
+    B = batch or w.batch
+    roots = synth.root_tokens(B, w.V, w.seed + 1)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        r = oracle.table_step(ld, lt, roots, w.n, w.k, w.max_depth, NEG_INF)
+        roots = r.next_root.copy()
+    dt = time.perf_counter() - t0
+    return {"value": B * steps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{steps} steps of {B} sequences (build + mask + verify), threshold off, no memo", "seconds": dt}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the same config and metric (rank 0 only)."""
+    if int(os.environ.get("RANK", 0)) != 0:
+        return
+    import oracle
+    oracle.build()
+    w = synth.WORKLOADS[args.workload]
+    ld, lt = synth.make_tables(w)
+    sample_b = 8                                        # bounded sample per step: 8 of the 32 sequences
+    steps, warm = max(1, min(args.steps, 4)), max(0, min(args.warmup, 1))
+    if warm:
+        cpu_baseline(w, ld, lt, warm, batch=sample_b)
+    cb = cpu_baseline(w, ld, lt, steps, batch=sample_b)
+    line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": int(args.gpus),
+            "steps": steps, "warmup": warm, "ms_per_step": cb["seconds"] * 1e3 / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{w.name}: V={w.V}, n={w.n}, k={w.k}, max_depth={w.max_depth}, delta=off; "
+                                   f"each step is a sample of {sample_b} of the batch's {w.batch} sequences"},
+            "cpu_baseline": {"value": cb["value"], "unit": UNIT, "cores": 1, "kind": "oracle", "sample": cb["sample"]},
+            "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="c4", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--delta", type=float, default=NEG_INF)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="ncu dram bytes per build call to report in roofline.traffic (from profiles/)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()
