@@ -1,5 +1,5 @@
 // Shared device helpers: ordered bf16 keys, mbarrier / bulk-copy wrappers with bounded
-// waits, deterministic block reductions.  sm_100a only.
+// waits, warp-level reductions.  sm_100a only.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -7,8 +7,13 @@
 
 namespace ot {
 
-constexpr int kThreads = 256;               // threads per CTA in every kernel of the library
-constexpr int kWarps = kThreads / 32;
+// CTA shape of the row pipeline: 8 consumer warps stream the logits, one producer warp feeds the
+// shared-memory ring, one finisher warp turns a finished row into probabilities and tree updates.
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumers = kConsumerWarps * 32;     // 256 consumer threads
+constexpr int kProducerWarp = kConsumerWarps;       // warp 8
+constexpr int kFinisherWarp = kConsumerWarps + 1;   // warp 9
+constexpr int kThreads = (kConsumerWarps + 2) * 32; // 320 threads per CTA
 constexpr int kMaxK = 32;
 constexpr int kMaxN = 256;
 
@@ -19,6 +24,11 @@ constexpr int kErrInternal = -5;
 __device__ __forceinline__ void set_status(int* status, int code) {
     atomicCAS(status, 0, code);             // keep the first error
 }
+
+// Every wait in the library is bounded by this many SM clock cycles (about two seconds); on
+// expiry the waiter records kErrTimeout in the status word and gives up, so a protocol error
+// ends as an error code, never as a hang.
+constexpr long long kWaitCycles = 1ll << 32;
 
 // ---------------------------------------------------------------------------------------------
 // bf16 bit pattern -> 16-bit key whose unsigned order equals the numeric order of the values
@@ -65,21 +75,28 @@ __device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
     asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
 }
-// d = a * b + c on two packed fp32 lanes.
-__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {
-    unsigned long long A, B, Cc, D;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(A) : "f"(a0), "f"(a1));
-    asm("mov.b64 %0, {%1, %1};" : "=l"(B) : "f"(b));
-    asm("mov.b64 %0, {%1, %1};" : "=l"(Cc) : "f"(c));
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(D) : "l"(A), "l"(B), "l"(Cc));
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(D));
+// Packed fp32 pairs (two lanes per instruction).
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
 }
-__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
-    unsigned long long A, B, D;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(A) : "f"(a0), "f"(a1));
-    asm("mov.b64 %0, {%1, %2};" : "=l"(B) : "f"(b0), "f"(b1));
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(D) : "l"(A), "l"(B));
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(D));
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+__device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
 // --- mbarrier + 1-D bulk async copy (global -> this CTA's shared memory, no multicast) ---
@@ -88,6 +105,9 @@ __device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t coun
 }
 __device__ __forceinline__ void mbar_fence_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
@@ -104,70 +124,73 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after kWaitLimit polls (each poll itself blocks for a hardware-defined
-// time slice), records a timeout in the status word and returns false.
-constexpr uint32_t kWaitLimit = 1u << 22;
+// Bounded wait by one thread; returns false (status set) when kWaitCycles pass without completion.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, int* status) {
-    for (uint32_t it = 0; it < kWaitLimit; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
-    set_status(status, kErrTimeout);
-    return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitCycles) { set_status(status, kErrTimeout); return false; }
+    }
+    return true;
+}
+// Whole-warp wait: lane 0 polls, the result is broadcast (the other lanes issue nothing meanwhile).
+__device__ __forceinline__ bool mbar_wait_warp(unsigned long long* bar, uint32_t parity, int* status) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, status) ? 1 : 0;
+    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+}
+
+// --- global-memory flags and queue words (gpu scope) ---
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_s32(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_s32(int* p, int v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 // ---------------------------------------------------------------------------------------------
-// Deterministic block reductions (fixed tree: lanes by xor-shuffle, then warps in order).
-// `scratch` needs kWarps entries; every thread gets the result.
+// Warp-level reductions / scans (fixed shuffle trees: deterministic).
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
     return v;
 }
-__device__ __forceinline__ double block_sum(double v, double* scratch) {
-    v = warp_sum(v);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-    __syncthreads();
-    double t = 0.0;
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) t += scratch[w];
-    return t;
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
 }
-__device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v, unsigned long long* scratch) {
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         unsigned long long u = __shfl_xor_sync(0xFFFFFFFFu, v, o);
         v = u > v ? u : v;
     }
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-    __syncthreads();
-    unsigned long long t = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) t = scratch[w] > t ? scratch[w] : t;
-    return t;
+    return v;
 }
-// Exclusive block scan of one int per thread (thread order); also returns the block total.
-__device__ __forceinline__ int block_excl_scan(int v, int* scratch /*kWarps*/, int& total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+__device__ __forceinline__ int warp_sum_i32(int v) { return __reduce_add_sync(0xFFFFFFFFu, v); }
+// Exclusive scan of one int per lane; total returned through `total`.
+__device__ __forceinline__ int warp_excl_scan(int v, int& total) {
+    const int lane = threadIdx.x & 31;
     int inc = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         int u = __shfl_up_sync(0xFFFFFFFFu, inc, o);
         if (lane >= o) inc += u;
     }
-    __syncthreads();
-    if (lane == 31) scratch[warp] = inc;
-    __syncthreads();
-    int base = 0, tot = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        int s = scratch[w];
-        if (w < warp) base += s;
-        tot += s;
-    }
-    total = tot;
-    return base + inc - v;
+    total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+    return inc - v;
 }
 
 }  // namespace ot

@@ -8,11 +8,13 @@
 #include <stdio.h>
 #include <string.h>
 
+#include "pipeline.cuh"
 #include "select.cuh"
 
 namespace ot {
 
 constexpr int kRowMul = 31;                 // row of (token t, depth d) = (t*31 + d) mod H
+constexpr int kSmallThreads = 256;          // block size of the mask / verify / init kernels
 
 __device__ __forceinline__ int row_of(int token, int depth, int H) {
     return (int)(((long long)token * kRowMul + depth) % H);
@@ -31,6 +33,9 @@ struct Workspace {
     int32_t* R;            // [B][2][n]
     double* E_prev;        // [B]
     int32_t* st;           // [B][8]
+    // work queue of the build: one item per (sequence, layer, frontier slot)
+    unsigned long long* q_items;   // [q_capacity]
+    int32_t* q_ctl;        // [8]  0: head (next to claim), 1: tail (published), 2: sequences finished, 3: all done
     // verify
     int32_t* g;            // [B][n+1]  target argmax after the root (0) and after node i (i+1)
     int32_t* vdone;        // [B]
@@ -42,6 +47,17 @@ struct Workspace {
     uint64_t* o_mask; int32_t* o_pos;
     int32_t *o_alen, *o_atok, *o_anode, *o_next;
 };
+enum { kQHead = 0, kQTail = 1, kQFinished = 2, kQDone = 3 };
+
+constexpr int kQueueMargin = 4096;          // room for one over-claim per resident CTA
+
+static size_t max_items(const opt_tree_config& c) {
+    const size_t n = c.n, kk = c.k < c.V ? c.k : c.V, Dcap = c.max_depth < c.n ? c.max_depth : c.n;
+    size_t per_seq = 1;
+    if (Dcap >= 2) per_seq += kk < n ? kk : n;
+    if (Dcap >= 3) per_seq += (Dcap - 2) * n;
+    return per_seq * (size_t)c.max_batch;
+}
 
 struct Layout {
     size_t total = 0;
@@ -65,6 +81,8 @@ static size_t carve(const opt_tree_config& c, char* base, Workspace* w) {
     OT_TAKE(R, int32_t, B * 2 * n)
     OT_TAKE(E_prev, double, B)
     OT_TAKE(st, int32_t, B * 8)
+    OT_TAKE(q_items, unsigned long long, max_items(c) + kQueueMargin)
+    OT_TAKE(q_ctl, int32_t, 8)
     OT_TAKE(g, int32_t, B * (n + 1))
     OT_TAKE(vdone, int32_t, B)
     OT_TAKE(status, int32_t, 1)
@@ -87,10 +105,11 @@ static size_t carve(const opt_tree_config& c, char* base, Workspace* w) {
     return (L.total + 255) & ~(size_t)255;
 }
 
-struct Params {            // by-value kernel parameters common to the build kernels
-    int V, H, n, k, kk, Dcap, max_depth;
+struct Params {            // by-value kernel parameters
+    int V, H, n, k, kk, Dcap, max_depth, B;
     float delta;
     int aligned;
+    int q_capacity;
 };
 
 __device__ __forceinline__ SeqWork seq_work(const Workspace& w, const Params& p, int b) {
@@ -118,99 +137,137 @@ __device__ __forceinline__ TreeOut tree_out(const opt_tree_out& o, const Params&
     return t;
 }
 
-__device__ __forceinline__ void init_barriers(BlockSmem& s) {
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) mbar_init(&s.full_bar[i], 1);
-        mbar_fence_init();
-    }
-    __syncthreads();
+// Queue item: bit 63 valid | b (15 bits) | layer d | rows in the layer | frontier slot (16 bits each).
+__device__ __forceinline__ unsigned long long item_encode(int b, int d, int fsize, int slot) {
+    return (1ull << 63) | ((unsigned long long)b << 48) | ((unsigned long long)d << 32) |
+           ((unsigned long long)fsize << 16) | (unsigned long long)slot;
 }
 
 // ------------------------------------------------------------------------------------------------
 // Kernels
 // ------------------------------------------------------------------------------------------------
-__global__ void init_build_kernel(Workspace w, int B) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= B) return;
-    int32_t* st = w.st + (size_t)b * 8;
-    st[kStFsize] = 1; st[kStActive] = 1; st[kStDone] = 0; st[kStNR] = 0; st[kStDepth] = 0;
-    w.E_prev[b] = 0.0;
+// Clears the queue, publishes one root row per sequence and resets the per-sequence state.
+__global__ void init_build_kernel(Workspace w, Params p) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < p.q_capacity) w.q_items[i] = i < p.B ? item_encode(i, 1, 1, 0) : 0ull;
+    if (i < p.B) {
+        int32_t* st = w.st + (size_t)i * 8;
+        st[kStFsize] = 1; st[kStDone] = 0; st[kStNR] = 0;
+        w.E_prev[i] = 0.0;
+    }
+    if (i == 0) { w.q_ctl[kQHead] = 0; w.q_ctl[kQTail] = p.B; w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; }
 }
 
-// One drafting step (layer d) of Algorithm 1: CTA (slot, b) expands frontier node `slot` of
-// sequence b; the CTA that finishes a sequence's last row also selects the layer.
-__global__ void __launch_bounds__(kThreads)
-build_round_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, const int32_t* __restrict__ root_token,
-                   opt_tree_out out, int d) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    BlockSmem& s = *reinterpret_cast<BlockSmem*>(smem_raw);
-    const int b = blockIdx.y, slot = blockIdx.x, tid = threadIdx.x;
-    const SeqWork sw = seq_work(w, p, b);
-    if (!__ldcg(&sw.st[kStActive])) return;
-    const int fsize = __ldcg(&sw.st[kStFsize]);
-    if (slot >= fsize) return;
-    init_barriers(s);
-
-    int token, depth;
-    double parent_phat;
-    if (d == 1) {
-        token = root_token[b]; depth = 0; parent_phat = 1.0;       // the root counts as factor 1 (Eq. 2)
-    } else {
-        const int gid = (d - 2) * p.n + slot;
-        token = __ldcg(&sw.T_tok[gid]); depth = d - 1; parent_phat = __ldcg(&sw.T_phat[gid]);
-    }
-    if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
-    const uint16_t* row = draft + (size_t)row_of(token, depth, p.H) * p.V;
-
-    uint32_t parity = 0;
-    RowResult res;
-    const bool ok = row_softmax_topk(s, row, p.V, p.k, p.aligned != 0, parity, w.status, res);
-    if (tid < p.k) {
-        double ph = -1.0; int32_t tk = -1;
-        if (ok && tid < res.kk) {
-            const unsigned long long key = s.win[tid];
-            tk = (int32_t)cand_token(key);
-            ph = parent_phat * (exp((double)cand_logit(key) - res.m) / res.S);   // Eq. 2
+// Source of the tree build: rows come from the global work queue.
+struct BuildSource {
+    Workspace w; Params p;
+    const uint16_t* draft; const int32_t* root_token;
+    __device__ bool next(RowDesc& d) {
+        const int idx = atomicAdd(&w.q_ctl[kQHead], 1);
+        if (idx >= p.q_capacity) return false;
+        unsigned long long item = ld_acquire_u64(&w.q_items[idx]);
+        if (!(item >> 63)) {
+            const long long t0 = clock64();
+            for (;;) {
+                if (ld_acquire_s32(&w.q_ctl[kQDone])) return false;
+                item = ld_acquire_u64(&w.q_items[idx]);
+                if (item >> 63) break;
+                if (clock64() - t0 > kWaitCycles) { set_status(w.status, kErrTimeout); return false; }
+                __nanosleep(64);
+            }
         }
-        sw.cand_phat[slot * p.k + tid] = ph;
-        sw.cand_tok[slot * p.k + tid] = tk;
+        d.b = (int)((item >> 48) & 0x7FFFu); d.d = (int)((item >> 32) & 0xFFFFu);
+        d.fsize = (int)((item >> 16) & 0xFFFFu); d.slot = (int)(item & 0xFFFFu);
+        int token, depth;
+        if (d.d == 1) { token = root_token[d.b]; depth = 0; }
+        else { token = __ldcg(&w.T_tok[(size_t)d.b * p.max_depth * p.n + (size_t)(d.d - 2) * p.n + d.slot]); depth = d.d - 1; }
+        if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
+        d.row = draft + (size_t)row_of(token, depth, p.H) * p.V;
+        return true;
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s.flag = (atomicAdd(&sw.st[kStDone], 1) == fsize - 1);
-    __syncthreads();
-    if (!s.flag) return;
-    __threadfence();
-    finish_layer(s, sw, tree_out(out, p, b), d, p.n, p.k, p.kk, p.Dcap, p.max_depth, p.delta);
+};
+
+// Sink of the tree build: candidates' path values (Eq. 2), then, for the row that completes its
+// layer, the layer selection / loop test, and either new queue items or the packed tree.
+struct BuildSink {
+    CtaSmem* s; Workspace w; Params p; opt_tree_out out;
+    __device__ void row_done(const RowDesc& d, const RowOut& r) {
+        const int lane = threadIdx.x & 31;
+        const SeqWork sw = seq_work(w, p, d.b);
+        const double parent_phat = d.d == 1 ? 1.0 : __ldcg(&sw.T_phat[(size_t)(d.d - 2) * p.n + d.slot]);   // root: factor 1
+        if (lane < p.k) {
+            sw.cand_phat[d.slot * p.k + lane] = lane < r.kk ? parent_phat * r.p : -1.0;
+            sw.cand_tok[d.slot * p.k + lane] = r.tok;
+        }
+        __threadfence();
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) last = atomicAdd(&sw.st[kStDone], 1) == d.fsize - 1;
+        last = __shfl_sync(0xFFFFFFFFu, last, 0);
+        if (!last) return;
+        __threadfence();
+        const int nl = finish_layer_warp(*s, sw, tree_out(out, p, d.b), d.d, p.n, p.k, p.kk, p.Dcap, p.max_depth, p.delta, w.status);
+        __threadfence();
+        __syncwarp();
+        if (nl > 0) {
+            int pos = 0;
+            if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
+            pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
+            for (int i = lane; i < nl; i += 32) {
+                if (pos + i < p.q_capacity) st_release_u64(&w.q_items[pos + i], item_encode(d.b, d.d + 1, nl, i));
+                else set_status(w.status, kErrInternal);
+            }
+        } else if (lane == 0) {
+            if (atomicAdd(&w.q_ctl[kQFinished], 1) == p.B - 1) st_release_s32(&w.q_ctl[kQDone], 1);
+        }
+    }
+};
+
+// Algorithm 1 for a whole batch in one launch: persistent CTAs pull rows from the queue; layers
+// of different sequences overlap freely because sequences never exchange data.
+__global__ void __launch_bounds__(kThreads)
+build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, const int32_t* __restrict__ root_token, opt_tree_out out) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
+    BuildSource src{w, p, draft, root_token};
+    BuildSink sink{&s, w, p, out};
+    run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, w.status);
 }
 
-// The row step alone, one CTA per listed row.
+// The row step alone over a list of rows (static round-robin over the CTAs).
+struct ListSource {
+    const uint16_t* logits; const int32_t* rows; int nrows, V, H, next_idx, stride; int* status;
+    __device__ bool next(RowDesc& d) {
+        if (next_idx >= nrows) return false;
+        int r = rows[next_idx];
+        if (r < 0 || r >= H) { set_status(status, kErrInternal); r = 0; }
+        d.row = logits + (size_t)r * V; d.slot = next_idx; d.b = d.d = 0; d.fsize = 1;
+        next_idx += stride;
+        return true;
+    }
+};
+struct ListSink {
+    int32_t* tok_out; double* prob_out; int k;
+    __device__ void row_done(const RowDesc& d, const RowOut& r) {
+        const int lane = threadIdx.x & 31;
+        if (lane < k) {
+            tok_out[(size_t)d.slot * k + lane] = r.tok;
+            prob_out[(size_t)d.slot * k + lane] = r.p;
+        }
+    }
+};
 __global__ void __launch_bounds__(kThreads)
-row_topk_kernel(Params p, const uint16_t* __restrict__ logits, const int32_t* __restrict__ rows,
+row_topk_kernel(Params p, const uint16_t* __restrict__ logits, const int32_t* __restrict__ rows, int nrows,
                 int32_t* tok_out, double* prob_out, int* status) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    BlockSmem& s = *reinterpret_cast<BlockSmem*>(smem_raw);
-    init_barriers(s);
-    int r = rows[blockIdx.x];
-    if (r < 0 || r >= p.H) { set_status(status, kErrInternal); r = 0; }
-    uint32_t parity = 0;
-    RowResult res;
-    const bool ok = row_softmax_topk(s, logits + (size_t)r * p.V, p.V, p.k, p.aligned != 0, parity, status, res);
-    const int tid = threadIdx.x;
-    if (tid < p.k) {
-        double pr = 0.0; int32_t tk = -1;
-        if (ok && tid < res.kk) {
-            const unsigned long long key = s.win[tid];
-            tk = (int32_t)cand_token(key);
-            pr = exp((double)cand_logit(key) - res.m) / res.S;
-        }
-        tok_out[(size_t)blockIdx.x * p.k + tid] = tk;
-        prob_out[(size_t)blockIdx.x * p.k + tid] = pr;
-    }
+    CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
+    ListSource src{logits, rows, nrows, p.V, p.H, (int)blockIdx.x, (int)gridDim.x, status};
+    ListSink sink{tok_out, prob_out, p.k};
+    run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, status);
 }
 
 // Tree attention mask + position ids: one CTA per sequence, one thread per node.
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kSmallThreads)
 mask_kernel(const int32_t* __restrict__ parent, const int32_t* __restrict__ depth, const int32_t* __restrict__ n_sel,
             const int32_t* __restrict__ base_pos, int n, uint64_t* mask, int32_t* position_ids, int* status) {
     const int b = blockIdx.x, i = threadIdx.x;
@@ -246,7 +303,7 @@ __device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
 }
 
 struct VerifySmem {
-    unsigned long long red_u64[kWarps];
+    unsigned long long red_u64[kSmallThreads / 32];
     int flag;
     int hit;
 };
@@ -254,7 +311,7 @@ struct VerifySmem {
 // Greedy verification.  CTA (j, b): j = 0 takes the target row after the root, j >= 1 the row after
 // kept node j-1; each finds the row's argmax (lowest token on ties).  The last CTA of a sequence
 // then walks the tree: accept the child that carries the target's token, until none does.
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kSmallThreads)
 verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const int32_t* __restrict__ root_token,
               opt_tree_out tree, int32_t* accept_len, int32_t* accept_tokens, int32_t* accept_nodes, int32_t* next_root) {
     __shared__ VerifySmem s;
@@ -275,18 +332,18 @@ verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const 
         float best = -INFINITY;
         int best_v = -1;
         int v = tid;
-        for (; v + 3 * kThreads < nv; v += 4 * kThreads) {
+        for (; v + 3 * kSmallThreads < nv; v += 4 * kSmallThreads) {
             uint4 q[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) q[u] = ld_nc_v4(vec + v + u * kThreads);
+            for (int u = 0; u < 4; ++u) q[u] = ld_nc_v4(vec + v + u * kSmallThreads);
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const uint32_t m2 = max_bf16x2(max_bf16x2(q[u].x, q[u].y), max_bf16x2(q[u].z, q[u].w));
                 const float f = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
-                if (f > best || best_v < 0) { best = f; best_v = v + u * kThreads; }
+                if (f > best || best_v < 0) { best = f; best_v = v + u * kSmallThreads; }
             }
         }
-        for (; v < nv; v += kThreads) {
+        for (; v < nv; v += kSmallThreads) {
             const uint4 q = ld_nc_v4(vec + v);
             const uint32_t m2 = max_bf16x2(max_bf16x2(q.x, q.y), max_bf16x2(q.z, q.w));
             const float f = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
@@ -302,17 +359,21 @@ verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const 
             }
         }
     } else {
-        for (int v = tid; v < p.V; v += kThreads) {
+        for (int v = tid; v < p.V; v += kSmallThreads) {
             const unsigned long long key = cand_key(__ldg(row + v), (uint32_t)v);
             best_key = key > best_key ? key : best_key;
         }
     }
-    best_key = block_max_u64(best_key, s.red_u64);
-    int32_t* g = w.g + (size_t)b * (p.n + 1);
-    if (tid == 0) g[j] = (int32_t)cand_token(best_key);
-    __threadfence();
+    best_key = warp_max_u64(best_key);
+    if ((tid & 31) == 0) s.red_u64[tid >> 5] = best_key;
     __syncthreads();
-    if (tid == 0) s.flag = (atomicAdd(&w.vdone[b], 1) == ns);
+    int32_t* g = w.g + (size_t)b * (p.n + 1);
+    if (tid == 0) {
+        for (int q = 1; q < kSmallThreads / 32; ++q) best_key = s.red_u64[q] > best_key ? s.red_u64[q] : best_key;
+        g[j] = (int32_t)cand_token(best_key);
+        __threadfence();
+        s.flag = (atomicAdd(&w.vdone[b], 1) == ns);
+    }
     __syncthreads();
     if (!s.flag) return;
     __threadfence();
@@ -320,8 +381,8 @@ verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const 
     // acceptance walk (block-wide child search; children of one node carry distinct tokens)
     int32_t* at = accept_tokens + (size_t)b * (p.max_depth + 1);
     int32_t* an = accept_nodes + (size_t)b * p.max_depth;
-    for (int i = tid; i <= p.max_depth; i += kThreads) at[i] = -1;
-    for (int i = tid; i < p.max_depth; i += kThreads) an[i] = -1;
+    for (int i = tid; i <= p.max_depth; i += kSmallThreads) at[i] = -1;
+    for (int i = tid; i < p.max_depth; i += kSmallThreads) an[i] = -1;
     __syncthreads();
     int cur = -1, A = 0;
     for (int step = 0; step <= p.max_depth; ++step) {
@@ -330,7 +391,7 @@ verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const 
         ++A;
         __syncthreads();
         if (A > p.max_depth) break;
-        for (int i = tid; i < ns; i += kThreads)
+        for (int i = tid; i < ns; i += kSmallThreads)
             if (par[i] == cur && tok[i] == y) s.hit = i;
         __syncthreads();
         const int hit = s.hit;
@@ -357,6 +418,8 @@ struct opt_tree_ctx {
     void* base;
     size_t bytes;
     int device;
+    int grid;              // resident CTAs of the persistent kernels (SMs x occupancy)
+    int q_capacity;
     int64_t launches;
 };
 
@@ -368,6 +431,7 @@ bool valid_cfg(const opt_tree_config* c) {
 int supported_cfg(const opt_tree_config* c) {
     if (c->n > OPT_TREE_MAX_N || c->k > OPT_TREE_MAX_K || c->k > c->V) return OPT_TREE_ERR_UNSUPPORTED;
     if ((long long)c->V * 31 + c->max_depth > 2147483647LL) return OPT_TREE_ERR_UNSUPPORTED;
+    if (c->max_batch > 32767 || c->max_depth > 65535) return OPT_TREE_ERR_UNSUPPORTED;
     return OPT_TREE_OK;
 }
 ot::Params make_params(const opt_tree_ctx* ctx, const void* table, float delta) {
@@ -376,6 +440,8 @@ ot::Params make_params(const opt_tree_ctx* ctx, const void* table, float delta) 
     p.V = c.V; p.H = c.H; p.n = c.n; p.k = c.k; p.kk = c.k < c.V ? c.k : c.V;
     p.Dcap = c.max_depth < c.n ? c.max_depth : c.n;
     p.max_depth = c.max_depth;
+    p.B = 0;
+    p.q_capacity = ctx->q_capacity;
     p.delta = delta;
     p.aligned = ((reinterpret_cast<uintptr_t>(table) & 15u) == 0 && (c.V % 8) == 0) ? 1 : 0;
     return p;
@@ -411,11 +477,17 @@ int opt_tree_create(opt_tree_ctx** out, const opt_tree_config* cfg) {
         return OPT_TREE_ERR_CUDA;
     }
     ot::carve(*cfg, static_cast<char*>(ctx->base), &ctx->ws);
+    ctx->q_capacity = (int)(ot::max_items(*cfg) + ot::kQueueMargin);
     bool ok = cudaMemset(ctx->base, 0, ctx->bytes) == cudaSuccess;
-    ok = ok && cudaFuncSetAttribute(ot::build_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)sizeof(ot::BlockSmem)) == cudaSuccess;
+    ok = ok && cudaFuncSetAttribute(ot::build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)sizeof(ot::CtaSmem)) == cudaSuccess;
     ok = ok && cudaFuncSetAttribute(ot::row_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)sizeof(ot::BlockSmem)) == cudaSuccess;
+                                    (int)sizeof(ot::CtaSmem)) == cudaSuccess;
+    int per_sm = 0, sms = 0;
+    ok = ok && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ot::build_kernel, ot::kThreads, sizeof(ot::CtaSmem)) == cudaSuccess;
+    ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device) == cudaSuccess;
+    ctx->grid = per_sm * sms;
+    ok = ok && ctx->grid >= 1 && ctx->grid <= ot::kQueueMargin;
     if (!ok) {
         cudaGetLastError();
         cudaFree(ctx->base);
@@ -438,22 +510,19 @@ int opt_tree_build(opt_tree_ctx* ctx, const void* draft, const int32_t* root_tok
     if (!ctx || !draft || !root_token || bad_tree(out) || B < 1 || delta != delta) return OPT_TREE_ERR_INVALID_ARG;
     if (B > ctx->cfg.max_batch) return OPT_TREE_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const ot::Params p = make_params(ctx, draft, delta);
-    ot::init_build_kernel<<<(B + 255) / 256, 256, 0, st>>>(ctx->ws, B);
-    ctx->launches++;
-    for (int d = 1; d <= p.Dcap; ++d) {
-        const int width = d == 1 ? 1 : (d == 2 ? (p.kk < p.n ? p.kk : p.n) : p.n);   // largest possible frontier
-        ot::build_round_kernel<<<dim3(width, B), ot::kThreads, sizeof(ot::BlockSmem), st>>>(
-            ctx->ws, p, static_cast<const uint16_t*>(draft), root_token, *out, d);
-        ctx->launches++;
-    }
+    ot::Params p = make_params(ctx, draft, delta);
+    p.B = B;
+    ot::init_build_kernel<<<(ctx->q_capacity + 255) / 256, 256, 0, st>>>(ctx->ws, p);
+    ot::build_kernel<<<ctx->grid, ot::kThreads, sizeof(ot::CtaSmem), st>>>(
+        ctx->ws, p, static_cast<const uint16_t*>(draft), root_token, *out);
+    ctx->launches += 2;
     return check_launch();
 }
 
 int opt_tree_mask(opt_tree_ctx* ctx, const opt_tree_out* tree, int32_t B, const int32_t* base_pos, uint64_t* mask,
                   int32_t* position_ids, void* stream) {
     if (!ctx || bad_tree(tree) || !mask || !position_ids || B < 1 || B > ctx->cfg.max_batch) return OPT_TREE_ERR_INVALID_ARG;
-    ot::mask_kernel<<<B, ot::kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+    ot::mask_kernel<<<B, ot::kSmallThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         tree->parent, tree->depth, tree->n_sel, base_pos, ctx->cfg.n, mask, position_ids, ctx->ws.status);
     ctx->launches++;
     return check_launch();
@@ -465,7 +534,7 @@ int opt_tree_verify(opt_tree_ctx* ctx, const opt_tree_out* tree, const void* tar
         B < 1 || B > ctx->cfg.max_batch)
         return OPT_TREE_ERR_INVALID_ARG;
     const ot::Params p = make_params(ctx, target, 0.0f);
-    ot::verify_kernel<<<dim3(ctx->cfg.n + 1, B), ot::kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+    ot::verify_kernel<<<dim3(ctx->cfg.n + 1, B), ot::kSmallThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         ctx->ws, p, static_cast<const uint16_t*>(target), root_token, *tree, accept_len, accept_tokens, accept_nodes, next_root);
     ctx->launches++;
     return check_launch();
@@ -476,8 +545,9 @@ int opt_tree_row_softmax_topk(opt_tree_ctx* ctx, const void* logits, const int32
     if (!ctx || !logits || !rows || !tok_out || !prob_out || nrows < 0) return OPT_TREE_ERR_INVALID_ARG;
     if (nrows == 0) return OPT_TREE_OK;
     const ot::Params p = make_params(ctx, logits, 0.0f);
-    ot::row_topk_kernel<<<nrows, ot::kThreads, sizeof(ot::BlockSmem), static_cast<cudaStream_t>(stream)>>>(
-        p, static_cast<const uint16_t*>(logits), rows, tok_out, prob_out, ctx->ws.status);
+    const int grid = nrows < ctx->grid ? nrows : ctx->grid;
+    ot::row_topk_kernel<<<grid, ot::kThreads, sizeof(ot::CtaSmem), static_cast<cudaStream_t>(stream)>>>(
+        p, static_cast<const uint16_t*>(logits), rows, nrows, tok_out, prob_out, ctx->ws.status);
     ctx->launches++;
     return check_launch();
 }

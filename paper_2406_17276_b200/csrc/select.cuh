@@ -1,9 +1,9 @@
-// K2 / K3: layer selection (the n candidates of largest path value), running E_sub(T, n),
-// the loop test of Algorithm 1, and the scan-based tree packer.  All block-wide (kThreads).
+// K2 / K3 by one warp: layer selection (the n candidates of largest path value), running
+// E_sub(T, n), the loop test of Algorithm 1, and the scan-based tree packer.
 //
 // Selection never sorts: an 8-pass radix select on the 64-bit keys finds the threshold of the
-// "need" largest, then an ordered compaction (block scans) emits the kept elements in index
-// order, which is exactly the storage order the method wants (candidate-index order for a layer,
+// "need" largest, then an ordered compaction (ballot scans) emits the kept elements in index
+// order, which is exactly the storage order the method wants (candidate-index order for a layer;
 // (depth, slot) order for the running top-n, which is also the packed order of the final tree).
 #pragma once
 
@@ -16,80 +16,87 @@ __device__ __forceinline__ unsigned long long phat_key(double p) { return (unsig
 
 // Threshold of the `need` largest keys among keyf(0..N).  On return thr is that key and need_eq
 // how many of the elements equal to thr belong to the selection (lowest indices first).
-// Requires 1 <= need <= number of non-zero keys.
+// Requires 1 <= need <= number of non-zero keys.  Whole warp; hist has 256 ints.
 template <class KeyFn>
-__device__ void radix_select(KeyFn keyf, int N, int need, BlockSmem& s, unsigned long long& thr, int& need_eq) {
-    const int tid = threadIdx.x;
+__device__ void warp_radix_select(KeyFn keyf, int N, int need, int* hist, unsigned long long& thr, int& need_eq) {
+    const int lane = threadIdx.x & 31;
     unsigned long long prefix = 0ull, pmask = 0ull;
     for (int pass = 7; pass >= 0; --pass) {
-        s.hist[tid] = 0;
-        __syncthreads();
-        for (int i = tid; i < N; i += kThreads) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) hist[lane * 8 + j] = 0;
+        __syncwarp();
+        for (int i = lane; i < N; i += 32) {
             const unsigned long long key = keyf(i);
-            if ((key & pmask) == prefix) atomicAdd(&s.hist[(int)((key >> (8 * pass)) & 255ull)], 1);
+            if ((key & pmask) == prefix) atomicAdd(&hist[(int)((key >> (8 * pass)) & 255ull)], 1);
         }
-        __syncthreads();
-        if (tid < 32) {
-            // lane L owns bins [8L, 8L+8); suffix sums over lanes from the top
-            int c[8], mine = 0;
+        __syncwarp();
+        int c[8], mine = 0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) { c[j] = s.hist[8 * tid + j]; mine += c[j]; }
-            int incl = mine;
+        for (int j = 0; j < 8; ++j) { c[j] = hist[lane * 8 + j]; mine += c[j]; }
+        int incl = mine;                                   // suffix sums over lanes from the top
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
-                if (tid + o < 32) incl += u;
-            }
-            const int above = incl - mine;                 // elements in higher lanes' bins
-            if (above < need && need <= incl) {
-                int a = above, b = 7;
-                while (b > 0 && a + c[b] < need) { a += c[b]; --b; }
-                s.sel_bin = 8 * tid + b;
-                s.sel_need = need - a;
+        for (int o = 1; o < 32; o <<= 1) {
+            int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
+            if (lane + o < 32) incl += u;
+        }
+        const int above = incl - mine;
+        const bool here = above < need && need <= incl;
+        int bin = 0, nd = 0;
+        if (here) {
+            int a = above;
+            bin = lane * 8;
+#pragma unroll
+            for (int b = 7; b >= 0; --b) {                 // highest bin whose suffix count reaches need
+                if (nd == 0) {
+                    if (a + c[b] >= need) { bin = lane * 8 + b; nd = need - a; }
+                    else a += c[b];
+                }
             }
         }
-        __syncthreads();
-        prefix |= (unsigned long long)s.sel_bin << (8 * pass);
+        const int src = __ffs(__ballot_sync(0xFFFFFFFFu, here)) - 1;
+        bin = __shfl_sync(0xFFFFFFFFu, bin, src);
+        need = __shfl_sync(0xFFFFFFFFu, nd, src);
+        prefix |= (unsigned long long)bin << (8 * pass);
         pmask |= 0xFFull << (8 * pass);
-        need = s.sel_need;
+        __syncwarp();
     }
     thr = prefix;
     need_eq = need;
 }
 
 // Emits, in index order, the elements with key > thr and the first need_eq with key == thr.
-// emit(pos, i) is called once per kept element; returns the number kept.
+// emit(pos, i) is called once per kept element; returns the number kept.  Whole warp.
 template <class KeyFn, class EmitFn>
-__device__ int compact_selected(KeyFn keyf, int N, unsigned long long thr, int need_eq, BlockSmem& s, EmitFn emit) {
-    const int tid = threadIdx.x;
-    int eq_base = 0, take_base = 0;
-    for (int i0 = 0; i0 < N; i0 += kThreads) {
-        const int i = i0 + tid;
+__device__ int warp_compact_selected(KeyFn keyf, int N, unsigned long long thr, int need_eq, EmitFn emit) {
+    const int lane = threadIdx.x & 31;
+    const unsigned below = (1u << lane) - 1u;
+    int eq_seen = 0, taken = 0;
+    for (int i0 = 0; i0 < N; i0 += 32) {
+        const int i = i0 + lane;
         const unsigned long long key = i < N ? keyf(i) : 0ull;
         const bool eq = i < N && key == thr;
-        int tot;
-        const int eq_rank = eq_base + block_excl_scan(eq ? 1 : 0, s.red_i32, tot);
-        eq_base += tot;
-        const bool take = i < N && (key > thr || (eq && eq_rank < need_eq));
-        const int pos = take_base + block_excl_scan(take ? 1 : 0, s.red_i32, tot);
-        take_base += tot;
-        if (take) emit(pos, i);
+        const unsigned eqm = __ballot_sync(0xFFFFFFFFu, eq);
+        const bool take = i < N && (key > thr || (eq && eq_seen + __popc(eqm & below) < need_eq));
+        const unsigned tm = __ballot_sync(0xFFFFFFFFu, take);
+        if (take) emit(taken + __popc(tm & below), i);
+        eq_seen += __popc(eqm);
+        taken += __popc(tm);
     }
-    return take_base;
+    return taken;
 }
 
 // Per-sequence state and arrays in the workspace (device pointers already offset to the sequence).
 struct SeqWork {
-    double* cand_phat;     // [n*k]    path values of this round's candidates (Eq. 2), slot-major
+    double* cand_phat;     // [n*k]    path values of this layer's candidates (Eq. 2), slot-major
     int32_t* cand_tok;     // [n*k]
     int32_t* T_tok;        // [D*n]    drafted nodes, gid = (depth-1)*n + slot
     int32_t* T_par;        // [D*n]    slot of the parent in the previous layer
     double* T_phat;        // [D*n]
     int32_t* R;            // [2][n]   running top-n as gids in ascending order, double-buffered by layer parity
     double* E_prev;        // [1]      E of Algorithm 1
-    int32_t* st;           // [8]      0: frontier size, 1: active, 2: rows done this round, 3: |R|, 4: layers drafted
+    int32_t* st;           // [8]      0: frontier size, 1: rows finished in this layer, 2: |R|
 };
-enum { kStFsize = 0, kStActive = 1, kStDone = 2, kStNR = 3, kStDepth = 4 };
+enum { kStFsize = 0, kStDone = 1, kStNR = 2 };
 
 struct TreeOut {           // mirrors opt_tree_out, pointers offset to the sequence
     int32_t *token, *parent, *depth;
@@ -101,82 +108,96 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
 
 // After all rows of layer d (1-based) of one sequence are expanded: choose the layer, update the
 // running top-n and E_sub, apply the loop test, and pack the tree if the sequence is finished.
-// Returns true if the sequence continues with layer d+1.
-__device__ bool finish_layer(BlockSmem& s, const SeqWork& w, const TreeOut& out, int d, int n, int k, int kk,
-                             int Dcap, int max_depth, float delta) {
-    const int tid = threadIdx.x;
+// Whole finisher warp.  Returns the size of the new layer if the sequence continues with layer
+// d+1, or 0 if it is finished (outputs written).
+__device__ int finish_layer_warp(CtaSmem& s, const SeqWork& w, const TreeOut& out, int d, int n, int k, int kk,
+                                 int Dcap, int max_depth, float delta, int* status) {
+    const int lane = threadIdx.x & 31;
     const int fsize = __ldcg(&w.st[kStFsize]);
     const int nR_old = __ldcg(&w.st[kStNR]);
     const int N = fsize * k;
     const int nvalid = fsize * kk;
     const int nl = nvalid < n ? nvalid : n;
     const int gid0 = (d - 1) * n;
+    unsigned long long thr;
+    int need_eq;
 
     // --- next layer: the nl candidates of largest path value, stored in candidate-index order ---
-    auto ckey = [&](int i) -> unsigned long long {
-        return (i % k) < kk ? phat_key(__ldcg(&w.cand_phat[i])) : 0ull;
-    };
-    unsigned long long thr; int need_eq;
-    radix_select(ckey, N, nl, s, thr, need_eq);
-    compact_selected(ckey, N, thr, need_eq, s, [&](int pos, int i) {
+    auto emit_layer = [&](int pos, int i) {
         w.T_tok[gid0 + pos] = __ldcg(&w.cand_tok[i]);
         w.T_par[gid0 + pos] = i / k;
         w.T_phat[gid0 + pos] = __ldcg(&w.cand_phat[i]);
-    });
-    __syncthreads();
+    };
+    auto gkey = [&](int i) -> unsigned long long { return (i % k) < kk ? phat_key(__ldcg(&w.cand_phat[i])) : 0ull; };
+    if (N <= 1024) {                                      // stage the keys in shared memory
+        for (int i = lane; i < N; i += 32) s.keys[i] = gkey(i);
+        __syncwarp();
+        auto skey = [&](int i) -> unsigned long long { return s.keys[i]; };
+        warp_radix_select(skey, N, nl, s.hist, thr, need_eq);
+        warp_compact_selected(skey, N, thr, need_eq, emit_layer);
+    } else {
+        warp_radix_select(gkey, N, nl, s.hist, thr, need_eq);
+        warp_compact_selected(gkey, N, thr, need_eq, emit_layer);
+    }
+    __syncwarp();
 
     // --- E_sub(T, n): the n largest path values among the previous top-n and the new layer ---
     const int32_t* Rold = w.R + ((d - 1) & 1) * n;
     int32_t* Rnew = w.R + (d & 1) * n;
-    const int NR = nR_old + nl;
+    const int NR = nR_old + nl;                           // <= 2n <= 512
     const int nR = NR < n ? NR : n;
-    auto gid_of = [&](int i) -> int { return i < nR_old ? __ldcg(&Rold[i]) : gid0 + (i - nR_old); };
-    auto rkey = [&](int i) -> unsigned long long { return phat_key(__ldcg(&w.T_phat[gid_of(i)])); };
-    radix_select(rkey, NR, nR, s, thr, need_eq);
-    compact_selected(rkey, NR, thr, need_eq, s, [&](int pos, int i) { Rnew[pos] = gid_of(i); });
-    __syncthreads();
+    for (int i = lane; i < NR; i += 32) {
+        const int gid = i < nR_old ? __ldcg(&Rold[i]) : gid0 + (i - nR_old);
+        s.gids[i] = gid;
+        s.keys[i] = phat_key(__ldcg(&w.T_phat[gid]));
+    }
+    __syncwarp();
+    auto rkey = [&](int i) -> unsigned long long { return s.keys[i]; };
+    warp_radix_select(rkey, NR, nR, s.hist, thr, need_eq);
+    warp_compact_selected(rkey, NR, thr, need_eq, [&](int pos, int i) {
+        Rnew[pos] = s.gids[i];
+        s.vals[pos] = __longlong_as_double((long long)(s.keys[i] - 1ull));
+    });
+    __syncwarp();
     double part = 0.0;
-    for (int i = tid; i < nR; i += kThreads) part += __ldcg(&w.T_phat[__ldcg(&Rnew[i])]);
-    const double esub = block_sum(part, s.red_f64);
+    for (int i = lane; i < nR; i += 32) part += s.vals[i];
+    const double esub = warp_sum(part);                   // fixed order: lanes stride the packed order
     const double eprev = __ldcg(w.E_prev);
-    const bool more = d < Dcap && (esub - eprev > (double)delta);
-    if (out.esub_trace && tid == 0) out.esub_trace[d - 1] = esub;
-
-    if (tid == 0) {
+    const bool more = d < Dcap && (esub - eprev > (double)delta);     // loop test of Algorithm 1
+    if (out.esub_trace && lane == 0) out.esub_trace[d - 1] = esub;
+    if (lane == 0) {
         w.st[kStFsize] = nl;
         w.st[kStNR] = nR;
         w.st[kStDone] = 0;
-        w.st[kStDepth] = d;
-        w.st[kStActive] = more ? 1 : 0;
         *w.E_prev = esub;
     }
-    if (!more) {
-        // --- pack: T_opt = the running top-n, already in (depth, parent's index, sibling rank) order ---
-        if (out.esub_trace) for (int i = d + tid; i < max_depth; i += kThreads) out.esub_trace[i] = 0.0;
-        for (int i = tid; i < n; i += kThreads) {
-            int32_t tok = -1, par = -1, dep = 0;
-            double ph = 0.0;
-            if (i < nR) {
-                const int gid = __ldcg(&Rnew[i]);
-                dep = gid / n + 1;
-                tok = __ldcg(&w.T_tok[gid]);
-                ph = __ldcg(&w.T_phat[gid]);
-                if (dep > 1) {
-                    const int pg = (dep - 2) * n + __ldcg(&w.T_par[gid]);
-                    int lo = 0, hi = i;                          // the parent is packed before its child
-                    while (lo < hi) {
-                        const int mid = (lo + hi) >> 1;
-                        if (__ldcg(&Rnew[mid]) < pg) lo = mid + 1; else hi = mid;
-                    }
-                    par = lo;
+    if (more) return nl;
+
+    // --- pack: T_opt = the running top-n, already in (depth, parent's index, sibling rank) order ---
+    if (out.esub_trace) for (int i = d + lane; i < max_depth; i += 32) out.esub_trace[i] = 0.0;
+    for (int i = lane; i < n; i += 32) {
+        int32_t tok = -1, par = -1, dep = 0;
+        double ph = 0.0;
+        if (i < nR) {
+            const int gid = __ldcg(&Rnew[i]);
+            dep = gid / n + 1;
+            tok = __ldcg(&w.T_tok[gid]);
+            ph = s.vals[i];
+            if (dep > 1) {
+                const int pg = (dep - 2) * n + __ldcg(&w.T_par[gid]);
+                int lo = 0, hi = i;                        // the parent is packed before its child
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (__ldcg(&Rnew[mid]) < pg) lo = mid + 1; else hi = mid;
                 }
+                if (lo >= i || __ldcg(&Rnew[lo]) != pg) set_status(status, kErrInternal);   // closure violated
+                par = lo;
             }
-            out.token[i] = tok; out.parent[i] = par; out.depth[i] = dep; out.phat[i] = ph;
         }
-        if (tid == 0) { *out.n_sel = nR; *out.depth_reached = d; *out.expected_len = esub; }
+        out.token[i] = tok; out.parent[i] = par; out.depth[i] = dep; out.phat[i] = ph;
     }
-    __syncthreads();
-    return more;
+    if (lane == 0) { *out.n_sel = nR; *out.depth_reached = d; *out.expected_len = esub; }
+    return 0;
 }
 
 }  // namespace ot
