@@ -136,8 +136,13 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
 // Whole-warp wait: lane 0 polls, the result is broadcast (the other lanes issue nothing meanwhile).
 __device__ __forceinline__ bool mbar_wait_warp(unsigned long long* bar, uint32_t parity, int* status) {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, status) ? 1 : 0;
-    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+    const bool leader = (threadIdx.x & 31) == 0;
+    if (leader) ok = mbar_wait(bar, parity, status) ? 1 : 0;
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    // The phase is complete and cannot advance again before this warp releases it, so one
+    // try_wait per remaining lane succeeds at once; it gives every lane its own acquire.
+    if (ok && !leader) mbar_try_wait(bar, parity);
+    return ok != 0;
 }
 
 // --- global-memory flags and queue words (gpu scope) ---
