@@ -7,13 +7,17 @@
 
 namespace ot {
 
-// CTA shape of the row pipeline: 8 consumer warps stream the logits, one producer warp feeds the
-// shared-memory ring, one finisher warp turns a finished row into probabilities and tree updates.
-constexpr int kConsumerWarps = 8;
-constexpr int kConsumers = kConsumerWarps * 32;     // 256 consumer threads
-constexpr int kProducerWarp = kConsumerWarps;       // warp 8
-constexpr int kFinisherWarp = kConsumerWarps + 1;   // warp 9
-constexpr int kThreads = (kConsumerWarps + 2) * 32; // 320 threads per CTA
+// CTA shape of the row pipeline (one CTA per SM): 16 consumer warps stream the logits, an issuer
+// warp feeds the shared-memory ring, a fetcher warp obtains row descriptors ahead of time, and
+// several finisher warps (one row each, round robin) turn finished rows into probabilities and
+// tree updates.  A lone warp advances slowly next to 16 busy ones, hence several finishers.
+constexpr int kConsumerWarps = 16;
+constexpr int kConsumers = kConsumerWarps * 32;     // 512 consumer threads
+constexpr int kIssuerWarp = kConsumerWarps;         // warp 16
+constexpr int kFetcherWarp = kConsumerWarps + 1;    // warp 17
+constexpr int kFirstFinisherWarp = kConsumerWarps + 2;
+constexpr int kFinishers = 6;
+constexpr int kThreads = (kFirstFinisherWarp + kFinishers) * 32;   // 768 threads per CTA
 constexpr int kMaxK = 32;
 constexpr int kMaxN = 256;
 
@@ -89,6 +93,11 @@ __device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigne
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
     return d;
 }
+__device__ __forceinline__ unsigned long long mul2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 __device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
     unsigned long long d;
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
@@ -124,25 +133,23 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait by one thread; returns false (status set) when kWaitCycles pass without completion.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, int* status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitCycles) { set_status(status, kErrTimeout); return false; }
-    }
-    return true;
-}
-// Whole-warp wait: lane 0 polls, the result is broadcast (the other lanes issue nothing meanwhile).
+// Bounded wait, called by every lane of a converged warp (try_wait suspends the thread in hardware
+// for a while, so the loop turns over slowly; the clock is read only once in 256 turns).  Returns
+// false to the whole warp (status set) when kWaitCycles pass without completion.
 __device__ __forceinline__ bool mbar_wait_warp(unsigned long long* bar, uint32_t parity, int* status) {
-    int ok = 1;
-    const bool leader = (threadIdx.x & 31) == 0;
-    if (leader) ok = mbar_wait(bar, parity, status) ? 1 : 0;
-    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-    // The phase is complete and cannot advance again before this warp releases it, so one
-    // try_wait per remaining lane succeeds at once; it gives every lane its own acquire.
-    if (ok && !leader) mbar_try_wait(bar, parity);
-    return ok != 0;
+    if (mbar_try_wait(bar, parity)) return true;
+    long long t0 = 0;
+    int turns = 0;
+    bool ok = true;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++turns & 255) == 0) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitCycles) { ok = false; break; }
+        }
+    }
+    if (!ok) set_status(status, kErrTimeout);
+    return __all_sync(0xFFFFFFFFu, ok);
 }
 
 // --- global-memory flags and queue words (gpu scope) ---

@@ -137,22 +137,33 @@ __device__ __forceinline__ TreeOut tree_out(const opt_tree_out& o, const Params&
     return t;
 }
 
-// Queue item: bit 63 valid | b (15 bits) | layer d | rows in the layer | frontier slot (16 bits each).
-__device__ __forceinline__ unsigned long long item_encode(int b, int d, int fsize, int slot) {
-    return (1ull << 63) | ((unsigned long long)b << 48) | ((unsigned long long)d << 32) |
-           ((unsigned long long)fsize << 16) | (unsigned long long)slot;
+// Queue item: bit 63 valid | b (15 bits) | layer d (9) | rows in the layer (9) | frontier slot (8) |
+// table row of the node to expand (22).  Packing the row index spares the consumer of an item a
+// dependent load of the node's token.
+constexpr int kMaxTableRows = 1 << 22;
+__device__ __forceinline__ unsigned long long item_encode(int b, int d, int fsize, int slot, int row) {
+    return (1ull << 63) | ((unsigned long long)b << 48) | ((unsigned long long)d << 39) |
+           ((unsigned long long)fsize << 30) | ((unsigned long long)slot << 22) | (unsigned long long)row;
 }
 
 // ------------------------------------------------------------------------------------------------
 // Kernels
 // ------------------------------------------------------------------------------------------------
 // Clears the queue, publishes one root row per sequence and resets the per-sequence state.
-__global__ void init_build_kernel(Workspace w, Params p) {
+__global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restrict__ root_token) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < p.q_capacity) w.q_items[i] = i < p.B ? item_encode(i, 1, 1, 0) : 0ull;
+    if (i < p.q_capacity) {
+        unsigned long long item = 0ull;
+        if (i < p.B) {
+            int token = root_token[i];
+            if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
+            item = item_encode(i, 1, 1, 0, row_of(token, 0, p.H));
+        }
+        w.q_items[i] = item;
+    }
     if (i < p.B) {
         int32_t* st = w.st + (size_t)i * 8;
-        st[kStFsize] = 1; st[kStDone] = 0; st[kStNR] = 0;
+        st[kStDone] = 0; st[kStNR] = 0;
         w.E_prev[i] = 0.0;
     }
     if (i == 0) { w.q_ctl[kQHead] = 0; w.q_ctl[kQTail] = p.B; w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; }
@@ -161,7 +172,7 @@ __global__ void init_build_kernel(Workspace w, Params p) {
 // Source of the tree build: rows come from the global work queue.
 struct BuildSource {
     Workspace w; Params p;
-    const uint16_t* draft; const int32_t* root_token;
+    const uint16_t* draft;
     __device__ bool next(RowDesc& d) {
         const int idx = atomicAdd(&w.q_ctl[kQHead], 1);
         if (idx >= p.q_capacity) return false;
@@ -176,13 +187,11 @@ struct BuildSource {
                 __nanosleep(64);
             }
         }
-        d.b = (int)((item >> 48) & 0x7FFFu); d.d = (int)((item >> 32) & 0xFFFFu);
-        d.fsize = (int)((item >> 16) & 0xFFFFu); d.slot = (int)(item & 0xFFFFu);
-        int token, depth;
-        if (d.d == 1) { token = root_token[d.b]; depth = 0; }
-        else { token = __ldcg(&w.T_tok[(size_t)d.b * p.max_depth * p.n + (size_t)(d.d - 2) * p.n + d.slot]); depth = d.d - 1; }
-        if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
-        d.row = draft + (size_t)row_of(token, depth, p.H) * p.V;
+        d.b = (int)((item >> 48) & 0x7FFFu); d.d = (int)((item >> 39) & 0x1FFu);
+        d.fsize = (int)((item >> 30) & 0x1FFu); d.slot = (int)((item >> 22) & 0xFFu);
+        int row = (int)(item & 0x3FFFFFu);
+        if (row >= p.H) { set_status(w.status, kErrInternal); row = 0; }
+        d.row = draft + (size_t)row * p.V;
         return true;
     }
 };
@@ -191,7 +200,7 @@ struct BuildSource {
 // layer, the layer selection / loop test, and either new queue items or the packed tree.
 struct BuildSink {
     CtaSmem* s; Workspace w; Params p; opt_tree_out out;
-    __device__ void row_done(const RowDesc& d, const RowOut& r) {
+    __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch& f) {
         const int lane = threadIdx.x & 31;
         const SeqWork sw = seq_work(w, p, d.b);
         const double parent_phat = d.d == 1 ? 1.0 : __ldcg(&sw.T_phat[(size_t)(d.d - 2) * p.n + d.slot]);   // root: factor 1
@@ -206,7 +215,10 @@ struct BuildSink {
         last = __shfl_sync(0xFFFFFFFFu, last, 0);
         if (!last) return;
         __threadfence();
-        const int nl = finish_layer_warp(*s, sw, tree_out(out, p, d.b), d.d, p.n, p.k, p.kk, p.Dcap, p.max_depth, p.delta, w.status);
+        if (!layer_lock(s->layer, w.status)) return;
+        const int nl = finish_layer_warp(s->layer, f.hist, sw, tree_out(out, p, d.b), d.d, d.fsize, p.n, p.k, p.kk, p.Dcap,
+                                         p.max_depth, p.delta, w.status);
+        layer_unlock(s->layer);
         __threadfence();
         __syncwarp();
         if (nl > 0) {
@@ -214,7 +226,9 @@ struct BuildSink {
             if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
             pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
             for (int i = lane; i < nl; i += 32) {
-                if (pos + i < p.q_capacity) st_release_u64(&w.q_items[pos + i], item_encode(d.b, d.d + 1, nl, i));
+                int token = __ldcg(&sw.T_tok[(size_t)(d.d - 1) * p.n + i]);
+                if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
+                if (pos + i < p.q_capacity) st_release_u64(&w.q_items[pos + i], item_encode(d.b, d.d + 1, nl, i, row_of(token, d.d, p.H)));
                 else set_status(w.status, kErrInternal);
             }
         } else if (lane == 0) {
@@ -225,11 +239,11 @@ struct BuildSink {
 
 // Algorithm 1 for a whole batch in one launch: persistent CTAs pull rows from the queue; layers
 // of different sequences overlap freely because sequences never exchange data.
-__global__ void __launch_bounds__(kThreads)
-build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, const int32_t* __restrict__ root_token, opt_tree_out out) {
+__global__ void __launch_bounds__(kThreads, 1)
+build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, opt_tree_out out) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
-    BuildSource src{w, p, draft, root_token};
+    BuildSource src{w, p, draft};
     BuildSink sink{&s, w, p, out};
     run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, w.status);
 }
@@ -248,7 +262,7 @@ struct ListSource {
 };
 struct ListSink {
     int32_t* tok_out; double* prob_out; int k;
-    __device__ void row_done(const RowDesc& d, const RowOut& r) {
+    __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch&) {
         const int lane = threadIdx.x & 31;
         if (lane < k) {
             tok_out[(size_t)d.slot * k + lane] = r.tok;
@@ -256,7 +270,7 @@ struct ListSink {
         }
     }
 };
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 1)
 row_topk_kernel(Params p, const uint16_t* __restrict__ logits, const int32_t* __restrict__ rows, int nrows,
                 int32_t* tok_out, double* prob_out, int* status) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -431,7 +445,7 @@ bool valid_cfg(const opt_tree_config* c) {
 int supported_cfg(const opt_tree_config* c) {
     if (c->n > OPT_TREE_MAX_N || c->k > OPT_TREE_MAX_K || c->k > c->V) return OPT_TREE_ERR_UNSUPPORTED;
     if ((long long)c->V * 31 + c->max_depth > 2147483647LL) return OPT_TREE_ERR_UNSUPPORTED;
-    if (c->max_batch > 32767 || c->max_depth > 65535) return OPT_TREE_ERR_UNSUPPORTED;
+    if (c->max_batch > 32767 || c->max_depth > 65535 || c->H > ot::kMaxTableRows) return OPT_TREE_ERR_UNSUPPORTED;
     return OPT_TREE_OK;
 }
 ot::Params make_params(const opt_tree_ctx* ctx, const void* table, float delta) {
@@ -512,9 +526,9 @@ int opt_tree_build(opt_tree_ctx* ctx, const void* draft, const int32_t* root_tok
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     ot::Params p = make_params(ctx, draft, delta);
     p.B = B;
-    ot::init_build_kernel<<<(ctx->q_capacity + 255) / 256, 256, 0, st>>>(ctx->ws, p);
+    ot::init_build_kernel<<<(ctx->q_capacity + 255) / 256, 256, 0, st>>>(ctx->ws, p, root_token);
     ot::build_kernel<<<ctx->grid, ot::kThreads, sizeof(ot::CtaSmem), st>>>(
-        ctx->ws, p, static_cast<const uint16_t*>(draft), root_token, *out);
+        ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
     ctx->launches += 2;
     return check_launch();
 }

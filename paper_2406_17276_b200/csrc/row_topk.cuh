@@ -1,37 +1,48 @@
 // K1: fused row softmax + top-k over the vocabulary (the row step of Algorithm 1: the
 // children of a node are its k most probable next tokens; their probabilities feed Eq. 2).
 //
-// A row of V bf16 logits is read exactly once from global memory, as 16 KB chunks that a
-// producer warp streams into a shared-memory ring with 1-D bulk async copies.  The eight
-// consumer warps
-//   * scan the first chunk(s) of the row for per-thread maxima; the k-th largest of those is a
-//     lower bound tau of the row's k-th largest logit;
-//   * then make ONE fused pass over every chunk: a logit >= tau goes to a small candidate list
-//     (it may be a winner, and it certainly includes the row maximum), every other logit adds
-//     2^((x - tau) * log2 e) to an fp32 partial sum (packed fp32x2 FMA + ex2.approx);
-// and a finisher warp turns the candidate list and the partial sums into the row's result:
-// exact ranking of the candidates on (bf16 bits, token id), fp64 exponentials for the candidates,
-// fp64 combine of the bulk, probabilities of the k winners.
-// Rows whose candidate list overflows (heavy ties, mostly -inf rows, tiny V) are redone by the
-// finisher warp with an exact radix-select path that re-reads the row from global memory.
+// A row of V bf16 logits is read exactly once from HBM, as 32 KB chunks that the issuer warp
+// streams into a shared-memory ring with 1-D bulk async copies.
+//
+// The 16 consumer warps make ONE branch-free pass over every chunk.  A consumer thread owns a
+// fixed set of 16-byte vectors of the row (vector index = tid mod 512) and keeps, over the row,
+//   * the maximum of its logits (packed bf16x2 max),
+//   * the sum of 2^(x*log2e - E) over its logits, E an integer exponent >= its running maximum
+//     (raising E rescales the sum by an exact power of two), in packed fp32x2 FMA + ex2.approx.
+// Nothing in that pass depends on a threshold, so consecutive rows stream without a bubble.
+//
+// A finisher warp then turns the 512 per-thread (max, sum) pairs into the row's result:
+//   * tau = k-th largest per-thread maximum: a lower bound of the row's k-th largest logit, so
+//     every winner lives in a thread whose maximum is >= tau ("flagged", about k of 512);
+//   * the flagged threads' vectors are read again (they are still in L2): logits >= tau become
+//     candidates, the others are summed like the bulk;
+//   * candidates are ranked exactly on (bf16 bits, token id) and their exponentials taken in fp64;
+//     the unflagged threads' sums are combined in fp64; probabilities of the k winners follow.
+// Rows this cannot handle (fewer than k finite per-thread maxima, heavy ties, extreme magnitudes)
+// are redone by the finisher warp with an exact radix-select path that re-reads the whole row.
 #pragma once
 
 #include "common.cuh"
 
 namespace ot {
 
-constexpr int kChunkElems = 8192;                  // bf16 elements per stage (16 KB)
-constexpr int kChunkVecs = kChunkElems / 8;        // 16-byte vectors per stage
-constexpr int kVecPerThread = kChunkVecs / kConsumers;   // 4
-constexpr int kStages = 3;                         // ring depth (48 KB)
-constexpr int kCandCap = 512;                      // candidate list capacity per row
-constexpr int kDesc = 8;                           // row descriptors in flight (> kStages)
+constexpr int kVecPerThread = 4;                   // 16-byte vectors per consumer thread per chunk
+constexpr int kChunkVecs = kConsumers * kVecPerThread;   // 2048
+constexpr int kChunkElems = kChunkVecs * 8;        // 16384 bf16 elements per stage (32 KB)
+constexpr int kStages = 4;                         // ring depth (128 KB)
+constexpr int kSlots = kFinishers + 2;             // finished rows waiting for / held by finishers
+constexpr int kCandCap = 128;                      // candidate list capacity per row
+constexpr int kMaxFlag = 64;                       // flagged threads the fast finisher accepts
+constexpr int kDesc = 4;                           // row descriptors fetched ahead
+constexpr int kPerLane = kConsumers / 32;          // per-thread results one finisher lane handles (16)
 
 constexpr float kLog2e = 1.44269504088896340736f;
 constexpr double kLog2eD = 1.44269504088896340736;
 constexpr double kFixScale = 4503599627370496.0;   // 2^52: fixed-point unit of the candidate terms
+constexpr float kExpFloor = -16000.0f;             // exponent of a thread that has seen no finite logit
+constexpr int kExpLimit = 15000;                   // |E| beyond this: magnitudes the fp32 pass cannot scale
 
-// Producer -> consumers: which row the next chunks of the stream belong to.
+// Fetcher -> issuer / consumers: which row the next chunks of the stream belong to.
 struct RowDesc {
     const uint16_t* row;      // global address of the row's first logit
     int b, d, slot;           // caller's coordinates (sequence, layer, frontier slot / list index)
@@ -39,120 +50,90 @@ struct RowDesc {
     int stop;                 // 1: no more rows, shut the pipeline down
 };
 
-// Consumers -> finisher: everything the fused pass leaves behind for one row.
+// Consumers -> finisher: what the fused pass leaves behind for one row.  Thread t's sum is
+// relative to the exponent of its warp, warpE[t / 32].
 struct RowSlot {
-    unsigned long long cand[kCandCap];     // candidate keys, unordered
-    double warp_part[kConsumerWarps];      // per-warp sums of 2^((x-tau)*log2e) over non-candidates
+    float tsum[kConsumers];
+    uint16_t tkey[kConsumers];     // per-thread maximum as an ordered key
+    int warpE[kConsumerWarps];
     RowDesc desc;
-    int cand_count;                        // may exceed kCandCap: overflow -> exact path
-    uint32_t tau_key;                      // ord16 of tau; <= kOrdNegInf -> exact path
+};
+
+struct FinScratch {                // private to one finisher warp
+    unsigned long long cand[kCandCap];         // candidate keys of the row in hand, unordered
+    int hist[256];
+    int flist[kMaxFlag];                       // flagged thread ids
+    int cand_count;
+};
+
+struct LayerScratch {              // shared by the finisher warps of a CTA under `lock`
+    unsigned long long keys[1024];             // staged candidate keys, then the keys of R + layer
+    unsigned long long lkeys[kMaxN];           // keys of the new layer, slot order
+    double vals[kMaxN];                        // path values of the new running top-n
+    int toks[1024];                            // staged candidate tokens
+    int gids[2 * kMaxN];
+    int rsel[kMaxN];                           // gids of the new running top-n, ascending
+    int lock;
 };
 
 struct alignas(128) CtaSmem {
     uint16_t stage[kStages][kChunkElems];
-    RowSlot slot[2];
+    RowSlot slot[kSlots];
+    FinScratch fin[kFinishers];
+    LayerScratch layer;
     RowDesc desc[kDesc];
-    unsigned long long full_bar[kStages];      // producer -> consumers (bulk copy landed)
-    unsigned long long empty_bar[kStages];     // consumers -> producer (stage may be overwritten)
-    unsigned long long ready_bar[2];           // consumers -> finisher (slot filled)
-    unsigned long long free_bar[2];            // finisher -> consumers (slot may be refilled)
-    uint32_t tmax[kConsumerWarps][32];
-    uint32_t tau_key;
-    // finisher scratch
-    unsigned long long keys[1024];
-    double vals[kMaxN];
-    int gids[2 * kMaxN];
-    int hist[256];
+    unsigned long long full_bar[kStages];      // issuer -> consumers (bulk copy landed)
+    unsigned long long empty_bar[kStages];     // consumers -> issuer (stage may be overwritten)
+    unsigned long long ready_bar[kSlots];      // consumers -> finisher (slot filled)
+    unsigned long long free_bar[kSlots];       // finisher -> consumers (slot may be refilled)
+    unsigned long long desc_full[kDesc];       // fetcher -> issuer (descriptor written)
+    unsigned long long desc_empty[kDesc];      // consumers -> fetcher (descriptor may be overwritten)
+    volatile int stop_row;                     // first row index that is the stop marker
 };
-
-// ---- k-th largest of one 16-bit key per consumer thread (k <= 32) ---------------------------
-__device__ __forceinline__ uint32_t warp_sort_desc(uint32_t v) {
-    const int lane = threadIdx.x & 31;
-#pragma unroll
-    for (int size = 2; size <= 32; size <<= 1) {
-#pragma unroll
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            uint32_t p = __shfl_xor_sync(0xFFFFFFFFu, v, stride);
-            bool keep_max = ((lane & stride) == 0) == ((lane & size) == 0);
-            v = keep_max ? max(v, p) : min(v, p);
-        }
-    }
-    return v;
-}
-// a, b sorted descending across lanes -> the 32 largest of both, sorted descending.
-__device__ __forceinline__ uint32_t warp_merge_top32(uint32_t a, uint32_t b) {
-    const int lane = threadIdx.x & 31;
-    uint32_t v = max(a, __shfl_sync(0xFFFFFFFFu, b, 31 - lane));
-#pragma unroll
-    for (int stride = 16; stride > 0; stride >>= 1) {
-        uint32_t p = __shfl_xor_sync(0xFFFFFFFFu, v, stride);
-        v = ((lane & stride) == 0) ? max(v, p) : min(v, p);
-    }
-    return v;
-}
-// Called by all consumer threads (named barrier 1).
-__device__ __forceinline__ uint32_t consumers_kth_largest(uint32_t key, int k, CtaSmem& s) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    s.tmax[warp][lane] = warp_sort_desc(key);
-    named_barrier_sync(1, kConsumers);
-    if (warp == 0) {
-        uint32_t v[kConsumerWarps];
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) v[w] = s.tmax[w][lane];
-#pragma unroll
-        for (int step = 1; step < kConsumerWarps; step <<= 1)
-#pragma unroll
-            for (int w = 0; w + step < kConsumerWarps; w += 2 * step) v[w] = warp_merge_top32(v[w], v[w + step]);
-        uint32_t kth = __shfl_sync(0xFFFFFFFFu, v[0], k - 1);
-        if (lane == 0) s.tau_key = kth;
-    }
-    named_barrier_sync(1, kConsumers);
-    return s.tau_key;
-}
 
 __device__ __forceinline__ int chunk_elems(int V, int c) {
     int rem = V - c * kChunkElems;
     return rem < kChunkElems ? rem : kChunkElems;
 }
 
-__device__ __forceinline__ void push_cand(RowSlot& slot, uint32_t bits, uint32_t token) {
-    int pos = atomicAdd(&slot.cand_count, 1);
-    if (pos < kCandCap) slot.cand[pos] = cand_key(bits, token);
+// ------------------------------------------------------------------------------------------------
+// Consumer side.
+// ------------------------------------------------------------------------------------------------
+struct ThreadAcc {                 // one consumer thread's running state over a row
+    unsigned long long acc0, acc1; // packed fp32 pairs
+    uint32_t pm;                   // packed bf16x2 running maximum
+    float E;                       // integer-valued exponent the sums are relative to
+    __device__ __forceinline__ void reset() { acc0 = 0ull; acc1 = 0ull; pm = 0xFF80FF80u; E = kExpFloor; }
+};
+
+__device__ __forceinline__ float pow2_float(int d) {            // 2^d for d <= 0; 0 below the normal range
+    return __int_as_float(max(d + 127, 0) << 23);
 }
 
-// Rare path of the fused pass: this thread's vectors of the chunk hold at least one candidate.
-__device__ __noinline__ float chunk_pass_slow(RowSlot& slot, uint4 w0, uint4 w1, uint4 w2, uint4 w3, uint32_t token_base,
-                                               int tid, float tau, float c_tau) {
-    static_assert(kVecPerThread == 4, "chunk_pass_slow takes four vectors");
-    float sum = 0.0f;
-#pragma unroll
-    for (int u = 0; u < kVecPerThread; ++u) {
-        const uint4 wu = u == 0 ? w0 : (u == 1 ? w1 : (u == 2 ? w2 : w3));
-        const uint32_t ww[4] = {wu.x, wu.y, wu.z, wu.w};
-        const uint32_t tok0 = token_base + (uint32_t)(tid + u * kConsumers) * 8u;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t bits = (i & 1) ? (ww[i >> 1] >> 16) : (ww[i >> 1] & 0xFFFFu);
-            const float x = bf16_bits_to_float(bits);
-            if (x >= tau) push_cand(slot, bits, tok0 + i);
-            else sum += ex2_approx(fmaf(x, kLog2e, c_tau));
-        }
-    }
-    return sum;
-}
-
-// Fused pass over this thread's share of one chunk (kVecPerThread vectors of 8 logits).
-__device__ __forceinline__ float chunk_pass(RowSlot& slot, const uint4* vec, int nv, uint32_t token_base, int tid,
-                                            float tau, float c_tau) {
+// This thread's share of one chunk (kVecPerThread vectors of 8 logits) folded into its state.
+__device__ __forceinline__ void chunk_pass(ThreadAcc& a, const uint4* vec, int nv, int tid) {
     uint4 w[kVecPerThread];
 #pragma unroll
     for (int u = 0; u < kVecPerThread; ++u) {
         const int v = tid + u * kConsumers;
         w[u] = v < nv ? vec[v] : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // -inf padding
     }
-    const unsigned long long L2 = pack2(kLog2e, kLog2e), C2 = pack2(c_tau, c_tau);
-    unsigned long long acc0 = 0ull, acc1 = 0ull;       // packed (0.0f, 0.0f)
-    float mx0 = -INFINITY, mx1 = -INFINITY;
+    // maximum of the 32 logits, then the exponent they are summed against
+    uint32_t m2 = 0xFF80FF80u;
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; ++u)
+        m2 = max_bf16x2(m2, max_bf16x2(max_bf16x2(w[u].x, w[u].y), max_bf16x2(w[u].z, w[u].w)));
+    a.pm = max_bf16x2(a.pm, m2);
+    const float f = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
+    float Ec;
+    asm("cvt.rpi.f32.f32 %0, %1;" : "=f"(Ec) : "f"(fminf(fmaxf(f * kLog2e, kExpFloor), -kExpFloor)));
+    const float En = fmaxf(a.E, Ec);
+    const float sc = pow2_float((int)(a.E - En));                    // exact: both are integers
+    const unsigned long long sc2 = pack2(sc, sc);
+    a.acc0 = mul2(a.acc0, sc2);
+    a.acc1 = mul2(a.acc1, sc2);
+    a.E = En;
+    const unsigned long long L2 = pack2(kLog2e, kLog2e), C2 = pack2(-En, -En);
 #pragma unroll
     for (int u = 0; u < kVecPerThread; ++u) {
         const uint32_t ww[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
@@ -160,33 +141,27 @@ __device__ __forceinline__ float chunk_pass(RowSlot& slot, const uint4* vec, int
         for (int i = 0; i < 4; ++i) {
             const float lo = __uint_as_float(ww[i] << 16), hi = __uint_as_float(ww[i] & 0xFFFF0000u);
             float a0, a1;
-            unpack2(fma2(pack2(lo, hi), L2, C2), a0, a1);            // (x - tau) * log2(e)
+            unpack2(fma2(pack2(lo, hi), L2, C2), a0, a1);            // x*log2e - E
             const unsigned long long e2 = pack2(ex2_approx(a0), ex2_approx(a1));
-            if (i & 1) { acc1 = add2(acc1, e2); mx1 = max3(mx1, lo, hi); }
-            else       { acc0 = add2(acc0, e2); mx0 = max3(mx0, lo, hi); }
+            if (i & 1) a.acc1 = add2(a.acc1, e2);
+            else       a.acc0 = add2(a.acc0, e2);
         }
     }
-    if (fmaxf(mx0, mx1) >= tau) return chunk_pass_slow(slot, w[0], w[1], w[2], w[3], token_base, tid, tau, c_tau);
-    float s0, s1;
-    unpack2(add2(acc0, acc1), s0, s1);
-    return s0 + s1;
 }
 
-// Per-thread packed maximum over this thread's share of one chunk (the sampling pass).
-__device__ __forceinline__ uint32_t chunk_max(const uint4* vec, int nv, int tid, uint32_t pm) {
-#pragma unroll
-    for (int u = 0; u < kVecPerThread; ++u) {
-        const int v = tid + u * kConsumers;
-        if (v < nv) {
-            const uint4 w = vec[v];
-            pm = max_bf16x2(max_bf16x2(pm, w.x), max_bf16x2(w.y, max_bf16x2(w.z, w.w)));
-        }
-    }
-    return pm;
+// End of a row: every thread's sum is brought to its warp's largest exponent and stored.
+__device__ __forceinline__ void store_thread_result(RowSlot& slot, const ThreadAcc& a, int tid) {
+    float s0, s1;
+    unpack2(add2(a.acc0, a.acc1), s0, s1);
+    const int e = (int)a.E;
+    const int ew = __reduce_max_sync(0xFFFFFFFFu, e);
+    slot.tsum[tid] = (s0 + s1) * pow2_float(e - ew);
+    slot.tkey[tid] = (uint16_t)max(ord16(a.pm & 0xFFFFu), ord16(a.pm >> 16));
+    if ((tid & 31) == 0) slot.warpE[tid >> 5] = ew;
 }
 
 // ------------------------------------------------------------------------------------------------
-// Finisher side (one warp).
+// Finisher side (one warp per row).
 // ------------------------------------------------------------------------------------------------
 struct RowOut {        // lane j < kk holds the j-th most probable token and its probability
     int kk;
@@ -194,10 +169,94 @@ struct RowOut {        // lane j < kk holds the j-th most probable token and its
     double p;
 };
 
+// 64 keys, two per lane (element i = lane + 32*q is x[q]), sorted descending by element index.
+__device__ __forceinline__ void warp_sort64_desc(unsigned long long& x0, unsigned long long& x1) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int size = 2; size <= 64; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            if (stride == 32) {
+                // partner of element lane is element lane+32; in the last merge all pairs keep the maximum low
+                const unsigned long long hi = x0 > x1 ? x0 : x1, lo = x0 > x1 ? x1 : x0;
+                x0 = hi; x1 = lo;
+            } else {
+                const unsigned long long p0 = __shfl_xor_sync(0xFFFFFFFFu, x0, stride);
+                const unsigned long long p1 = __shfl_xor_sync(0xFFFFFFFFu, x1, stride);
+                const bool lower = (lane & stride) == 0;
+                const bool desc0 = (lane & size) == 0;                   // block of element lane
+                const bool desc1 = ((lane + 32) & size) == 0;            // block of element lane+32
+                x0 = (lower == desc0) ? (x0 > p0 ? x0 : p0) : (x0 < p0 ? x0 : p0);
+                x1 = (lower == desc1) ? (x1 > p1 ? x1 : p1) : (x1 < p1 ? x1 : p1);
+            }
+        }
+    }
+}
+
+// 32 keys, one per lane, sorted descending across lanes.
+__device__ __forceinline__ unsigned long long warp_sort32_desc(unsigned long long v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const unsigned long long p = __shfl_xor_sync(0xFFFFFFFFu, v, stride);
+            const bool keep_max = ((lane & stride) == 0) == ((lane & size) == 0);
+            v = keep_max ? (v > p ? v : p) : (v < p ? v : p);
+        }
+    }
+    return v;
+}
+
+// k-th largest of the 16-bit keys key[0..kPerLane) held by every lane (32*kPerLane keys in all):
+// two 8-bit radix passes over a shared histogram.  1 <= k <= number of keys.
+__device__ __forceinline__ uint32_t warp_kth_largest16(const uint32_t (&key)[kPerLane], int k, int* hist) {
+    const int lane = threadIdx.x & 31;
+    uint32_t prefix = 0;
+    int need = k;
+#pragma unroll
+    for (int pass = 1; pass >= 0; --pass) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) hist[lane * 8 + j] = 0;
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j)
+            if (pass == 1 || (key[j] >> 8) == prefix) atomicAdd(&hist[(key[j] >> (8 * pass)) & 255u], 1);
+        __syncwarp();
+        int c[8], mine = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = hist[lane * 8 + j]; mine += c[j]; }
+        int incl = mine;                                   // suffix sums over lanes from the top
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
+            if (lane + o < 32) incl += u;
+        }
+        const int above = incl - mine;
+        const bool here = above < need && need <= incl;
+        int bin = 0, nd = 0;
+        if (here) {
+            int a = above;
+#pragma unroll
+            for (int b = 7; b >= 0; --b) {                 // highest bin whose suffix count reaches need
+                if (nd == 0) {
+                    if (a + c[b] >= need) { bin = lane * 8 + b; nd = need - a; }
+                    else a += c[b];
+                }
+            }
+        }
+        const int src = __ffs(__ballot_sync(0xFFFFFFFFu, here)) - 1;
+        bin = __shfl_sync(0xFFFFFFFFu, bin, src);
+        need = __shfl_sync(0xFFFFFFFFu, nd, src);
+        prefix = pass == 1 ? (uint32_t)bin : ((prefix << 8) | (uint32_t)bin);
+        __syncwarp();
+    }
+    return prefix;
+}
+
 // Exact path for one row by one warp: radix select on the 16-bit keys, ordered tie handling,
-// fp64 sum.  Leaves exactly kk candidates in slot.cand and returns the row maximum and sum.
-__device__ __noinline__ void row_exact_warp(CtaSmem& s, RowSlot& slot, const uint16_t* row, int V, int kk,
-                                            double& m_out, double& S_out) {
+// fp64 sum.  Leaves exactly kk candidates in f.cand and returns the row maximum and sum.
+__device__ __noinline__ void row_exact_warp(FinScratch& f, const uint16_t* row, int V, int kk, double& m_out, double& S_out) {
     const int lane = threadIdx.x & 31;
     uint32_t mk = 0;
     for (int v = lane; v < V; v += 32) mk = max(mk, ord16(__ldg(row + v)));
@@ -206,15 +265,15 @@ __device__ __noinline__ void row_exact_warp(CtaSmem& s, RowSlot& slot, const uin
     uint32_t prefix = 0, pmask = 0;
     int need = kk;
     for (int pass = 1; pass >= 0; --pass) {
-        for (int j = 0; j < 8; ++j) s.hist[lane * 8 + j] = 0;
+        for (int j = 0; j < 8; ++j) f.hist[lane * 8 + j] = 0;
         __syncwarp();
         for (int v = lane; v < V; v += 32) {
             const uint32_t key = ord16(__ldg(row + v));
-            if ((key & pmask) == prefix) atomicAdd(&s.hist[(key >> (8 * pass)) & 255u], 1);
+            if ((key & pmask) == prefix) atomicAdd(&f.hist[(key >> (8 * pass)) & 255u], 1);
         }
         __syncwarp();
         int c[8], mine = 0;
-        for (int j = 0; j < 8; ++j) { c[j] = s.hist[lane * 8 + j]; mine += c[j]; }
+        for (int j = 0; j < 8; ++j) { c[j] = f.hist[lane * 8 + j]; mine += c[j]; }
         int incl = mine;
         for (int o = 1; o < 32; o <<= 1) {
             int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
@@ -250,7 +309,7 @@ __device__ __noinline__ void row_exact_warp(CtaSmem& s, RowSlot& slot, const uin
         eq_seen += __popc(eqm);
         const bool take = valid && (key > thr || (key == thr && eq_rank < need));
         const unsigned tm = __ballot_sync(0xFFFFFFFFu, take);
-        if (take) slot.cand[count + __popc(tm & ((1u << lane) - 1u))] = cand_key(bits, (uint32_t)v);
+        if (take) f.cand[count + __popc(tm & ((1u << lane) - 1u))] = cand_key(bits, (uint32_t)v);
         count += __popc(tm);
         if (valid && key > kOrdNegInf) {
             if (bits != memo_bits) { memo_bits = bits; memo_e = exp((double)bf16_bits_to_float(bits) - m); }
@@ -258,59 +317,195 @@ __device__ __noinline__ void row_exact_warp(CtaSmem& s, RowSlot& slot, const uin
         }
     }
     __syncwarp();
-    if (lane == 0) slot.cand_count = count;
+    if (lane == 0) f.cand_count = count;
     __syncwarp();
     m_out = m;
     S_out = warp_sum(acc);
 }
 
-// Turns a finished slot into the row's k winners.  Whole finisher warp.
-__device__ __forceinline__ void finish_row_warp(CtaSmem& s, RowSlot& slot, int V, int k, RowOut& out) {
+// One 16-byte vector of the row (8 logits starting at token 8*vi) as four packed words; logits at or
+// beyond V read as -inf.  `aligned` rows take one vector load, others eight scalar loads.
+__device__ __forceinline__ uint4 load_row_vec(const uint16_t* row, int vi, int V, bool aligned) {
+    if (aligned) {
+        uint4 v;
+        asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(reinterpret_cast<const uint4*>(row) + vi));
+        return v;
+    }
+    uint32_t h[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) h[e] = (vi * 8 + e < V) ? (uint32_t)__ldg(row + vi * 8 + e) : 0xFF80u;
+    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+}
+
+// Turns a finished slot into the row's k winners.  Whole finisher warp; f is its private scratch.
+__device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& slot, int V, int k, bool aligned, RowOut& out) {
     const int lane = threadIdx.x & 31;
     const int kk = k < V ? k : V;
-    int M = slot.cand_count;
-    const uint32_t tau_key = slot.tau_key;
-    double m, S;
-    if (tau_key <= kOrdNegInf || M > kCandCap) {
-        row_exact_warp(s, slot, slot.desc.row, V, kk, m, S);
-        M = slot.cand_count;
-    } else {
-        unsigned long long best = 0ull;
-        for (int c = lane; c < M; c += 32) best = max(best, slot.cand[c]);
-        best = warp_max_u64(best);
-        m = (double)cand_logit(best);
-        unsigned long long fx = 0ull;
-        for (int c = lane; c < M; c += 32) fx += __double2ull_rn(exp((double)cand_logit(slot.cand[c]) - m) * kFixScale);
-        fx = warp_sum_u64(fx);                       // integer sum: independent of the push order
-        double bulk = 0.0;
+    const int nvec = (V + 7) >> 3;
+
+    // this lane's 16 consecutive threads all belong to consumer warp lane / 2
+    uint32_t key[kPerLane];
+    {
+        const uint4* kp = reinterpret_cast<const uint4*>(&slot.tkey[lane * kPerLane]);
 #pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) bulk += slot.warp_part[w];
-        // Bulk terms are 2^(x*L32 + c_tau) with c_tau = fl(-tau*L32); wanted e^(x-m) = 2^((x-m)*L).
-        // The exponent gap x*(L-L32) - m*L - c_tau is evaluated at a typical bulk logit x = tau - 2.
-        const float tau = bf16_bits_to_float(ord16_inv(tau_key));
-        const double c_tau = (double)(-tau * kLog2e);
-        const double gap = ((double)tau - 2.0) * (kLog2eD - (double)kLog2e) - m * kLog2eD - c_tau;
-        S = bulk * exp2(gap) + (double)fx / kFixScale;
-    }
-    // Selection by repeated warp argmax (all keys distinct).
-    unsigned long long lbest = 0ull, mine = 0ull;
-    int lidx = -1;
-    for (int c = lane; c < M; c += 32) { const unsigned long long key = slot.cand[c]; if (key > lbest) { lbest = key; lidx = c; } }
-    for (int j = 0; j < kk; ++j) {
-        const unsigned long long wbest = warp_max_u64(lbest);
-        if (lane == j) mine = wbest;
-        if (lbest == wbest && lidx >= 0) {           // this lane owned the winner: retire it and rescan
-            slot.cand[lidx] = 0ull;
-            lbest = 0ull; lidx = -1;
-            for (int c = lane; c < M; c += 32) { const unsigned long long key = slot.cand[c]; if (key > lbest) { lbest = key; lidx = c; } }
+        for (int q = 0; q < kPerLane / 8; ++q) {
+            const uint4 w = kp[q];
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { key[q * 8 + 2 * i] = ww[i] & 0xFFFFu; key[q * 8 + 2 * i + 1] = ww[i] >> 16; }
         }
     }
-    out.kk = kk;
-    out.tok = -1;
-    out.p = 0.0;
-    if (lane < kk) {
-        out.tok = (int32_t)cand_token(mine);
-        out.p = exp((double)cand_logit(mine) - m) / S;
+    const int myE = slot.warpE[lane >> 1];
+    const int emax = __reduce_max_sync(0xFFFFFFFFu, myE);
+    uint32_t mk = 0;
+#pragma unroll
+    for (int j = 0; j < kPerLane; ++j) mk = max(mk, key[j]);
+    mk = __reduce_max_sync(0xFFFFFFFFu, mk);
+
+    // tau: the kk-th largest per-thread maximum.  The maxima of a row lie close together, so a
+    // histogram with one bin per key value over the 256 values below the largest usually holds kk
+    // of them (and spreads the shared-memory atomics); otherwise two generic radix passes.
+    uint32_t tau_key;
+    {
+        const uint32_t base = mk > 255u ? mk - 255u : 0u;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) f.hist[lane * 8 + j] = 0;
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j)
+            if (key[j] >= base) atomicAdd(&f.hist[key[j] - base], 1);
+        __syncwarp();
+        int c[8], mine = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = f.hist[lane * 8 + j]; mine += c[j]; }
+        int incl = mine;                                   // suffix sums over lanes from the top
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
+            if (lane + o < 32) incl += u;
+        }
+        const int above = incl - mine;
+        const bool here = above < kk && kk <= incl;
+        int bin = -1;
+        if (here) {
+            int a = above;
+#pragma unroll
+            for (int b = 7; b >= 0; --b) {                 // highest bin whose suffix count reaches kk
+                if (bin < 0) {
+                    if (a + c[b] >= kk) bin = lane * 8 + b;
+                    else a += c[b];
+                }
+            }
+        }
+        const unsigned hm = __ballot_sync(0xFFFFFFFFu, here);
+        __syncwarp();
+        if (hm) tau_key = base + (uint32_t)__shfl_sync(0xFFFFFFFFu, bin, __ffs(hm) - 1);
+        else tau_key = warp_kth_largest16(key, kk, f.hist);
+    }
+    bool exact = tau_key <= kOrdNegInf || emax >= kExpLimit || emax <= -kExpLimit;
+
+    // bulk of the unflagged threads; flagged threads listed in thread order
+    uint32_t fmask = 0;
+    float part32 = 0.0f;
+    {
+        const float4* sp = reinterpret_cast<const float4*>(&slot.tsum[lane * kPerLane]);
+#pragma unroll
+        for (int q = 0; q < kPerLane / 4; ++q) {
+            const float4 t4 = sp[q];
+            const float tt[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const bool fl = key[q * 4 + i] >= tau_key;
+                fmask |= fl ? (1u << (q * 4 + i)) : 0u;
+                part32 += fl ? 0.0f : tt[i];
+            }
+        }
+    }
+    int nflag = 0;
+    if (!exact) {
+        const int base = warp_excl_scan(__popc(fmask), nflag);
+        if (nflag <= kMaxFlag) {
+            int pos = base;
+            for (uint32_t mm = fmask; mm; mm &= mm - 1) f.flist[pos++] = lane * kPerLane + (__ffs(mm) - 1);
+        } else {
+            exact = true;
+        }
+    }
+    if (lane == 0) f.cand_count = 0;
+    __syncwarp();
+
+    double m = (double)bf16_bits_to_float(ord16_inv(mk)), S = 0.0;
+    int M = 0;
+    if (!exact) {
+        const double part = (double)(part32 * pow2_float(myE - emax));
+        // flagged threads: read their vectors again, split candidates from bulk
+        const float tau_f = bf16_bits_to_float(ord16_inv(tau_key));
+        const int nchunks = (V + kChunkElems - 1) / kChunkElems;
+        const int vpt = nchunks * kVecPerThread;
+        const int total = nflag * vpt;
+        const float negE = -(float)emax;
+        float fb = 0.0f;
+        for (int i0 = 0; i0 < total; i0 += 32 * 4) {
+            uint4 w[4];
+            int vis[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int idx = i0 + u * 32 + lane;
+                vis[u] = -1;
+                if (idx < total) {
+                    const int fi = idx / vpt, j = idx - fi * vpt;
+                    const int vi = (j / kVecPerThread) * kChunkVecs + (j % kVecPerThread) * kConsumers + f.flist[fi];
+                    if (vi < nvec) { vis[u] = vi; w[u] = load_row_vec(slot.desc.row, vi, V, aligned); }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (vis[u] < 0) continue;
+                const uint32_t ww[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const uint32_t bits = (e & 1) ? (ww[e >> 1] >> 16) : (ww[e >> 1] & 0xFFFFu);
+                    const float x = bf16_bits_to_float(bits);
+                    if (x >= tau_f) {
+                        const int pos = atomicAdd(&f.cand_count, 1);
+                        if (pos < kCandCap) f.cand[pos] = cand_key(bits, (uint32_t)(vis[u] * 8 + e));
+                    } else {
+                        fb += ex2_approx(fmaf(x, kLog2e, negE));
+                    }
+                }
+            }
+        }
+        __syncwarp();
+        M = f.cand_count;
+        if (M > 64) exact = true;
+        else {
+            // Bulk terms are 2^(fl(x*L32) - E) with L32 the fp32 log2(e); wanted e^(x-m) = 2^((x-m)*L).
+            // The exponent gap E - m*L + x*(L - L32) is evaluated at a typical bulk logit x = tau - 2.
+            const double gap = (double)emax - m * kLog2eD + ((double)tau_f - 2.0) * (kLog2eD - (double)kLog2e);
+            S = warp_sum(part + (double)fb) * exp2(gap);
+        }
+    }
+    if (exact) {
+        row_exact_warp(f, slot.desc.row, V, kk, m, S);
+        M = f.cand_count;                                     // == kk <= 32
+    }
+    __syncwarp();
+
+    out.kk = kk; out.tok = -1; out.p = 0.0;
+    if (M <= 32) {
+        // one candidate per lane: sort, then every lane's exponential once
+        const unsigned long long mine = warp_sort32_desc(lane < M ? f.cand[lane] : 0ull);
+        const double e = lane < M ? exp((double)cand_logit(mine) - m) : 0.0;
+        if (!exact) S += (double)warp_sum_u64(__double2ull_rn(e * kFixScale)) / kFixScale;   // integer sum: order free
+        if (lane < kk) { out.tok = (int32_t)cand_token(mine); out.p = e / S; }
+    } else {
+        unsigned long long x0 = f.cand[lane], x1 = lane + 32 < M ? f.cand[lane + 32] : 0ull;
+        warp_sort64_desc(x0, x1);
+        const double e0 = exp((double)cand_logit(x0) - m);
+        const double e1 = x1 ? exp((double)cand_logit(x1) - m) : 0.0;
+        S += (double)warp_sum_u64(__double2ull_rn(e0 * kFixScale) + __double2ull_rn(e1 * kFixScale)) / kFixScale;
+        if (lane < kk) { out.tok = (int32_t)cand_token(x0); out.p = e0 / S; }
     }
 }
 

@@ -14,20 +14,39 @@ namespace ot {
 // Positive doubles order like their bit patterns; +1 keeps every valid key above the "invalid" key 0.
 __device__ __forceinline__ unsigned long long phat_key(double p) { return (unsigned long long)__double_as_longlong(p) + 1ull; }
 
-// Threshold of the `need` largest keys among keyf(0..N).  On return thr is that key and need_eq
-// how many of the elements equal to thr belong to the selection (lowest indices first).
+__device__ __forceinline__ unsigned long long warp_or_u64(unsigned long long v) {
+    const uint32_t lo = __reduce_or_sync(0xFFFFFFFFu, (uint32_t)v), hi = __reduce_or_sync(0xFFFFFFFFu, (uint32_t)(v >> 32));
+    return ((unsigned long long)hi << 32) | lo;
+}
+__device__ __forceinline__ unsigned long long warp_and_u64(unsigned long long v) {
+    const uint32_t lo = __reduce_and_sync(0xFFFFFFFFu, (uint32_t)v), hi = __reduce_and_sync(0xFFFFFFFFu, (uint32_t)(v >> 32));
+    return ((unsigned long long)hi << 32) | lo;
+}
+
+// Threshold of the `need` largest keys among keyf(0..N); key 0 means "not an element".
+// key_or / key_and are the bitwise OR / AND over all non-zero keys (the caller folds them into the
+// sweep that stages the keys): the bits on which all keys agree need no pass, and a pass whose
+// threshold bin holds exactly the elements still needed ends the search.  On return the selection
+// is {key > thr} plus the first need_eq elements (lowest indices) with key == thr.
 // Requires 1 <= need <= number of non-zero keys.  Whole warp; hist has 256 ints.
 template <class KeyFn>
-__device__ void warp_radix_select(KeyFn keyf, int N, int need, int* hist, unsigned long long& thr, int& need_eq) {
+__device__ void warp_radix_select(KeyFn keyf, int N, int need, int* hist, unsigned long long key_or,
+                                  unsigned long long key_and, unsigned long long& thr, int& need_eq) {
     const int lane = threadIdx.x & 31;
-    unsigned long long prefix = 0ull, pmask = 0ull;
-    for (int pass = 7; pass >= 0; --pass) {
+    const unsigned long long diff = key_or ^ key_and;
+    if (diff == 0ull) { thr = key_or; need_eq = need; return; }          // all elements equal
+    int top = 64 - __clzll((long long)diff);                             // the low `top` bits vary
+    unsigned long long prefix = top == 64 ? 0ull : ((key_or >> top) << top);
+    while (top > 0) {
+        const int wbits = top < 8 ? top : 8, shift = top - wbits;
+        const unsigned int dmask = (1u << wbits) - 1u;
 #pragma unroll
         for (int j = 0; j < 8; ++j) hist[lane * 8 + j] = 0;
         __syncwarp();
         for (int i = lane; i < N; i += 32) {
             const unsigned long long key = keyf(i);
-            if ((key & pmask) == prefix) atomicAdd(&hist[(int)((key >> (8 * pass)) & 255ull)], 1);
+            const bool match = key != 0ull && (top == 64 || (key >> top) == (prefix >> top));
+            if (match) atomicAdd(&hist[(int)((unsigned int)(key >> shift) & dmask)], 1);
         }
         __syncwarp();
         int c[8], mine = 0;
@@ -41,14 +60,14 @@ __device__ void warp_radix_select(KeyFn keyf, int N, int need, int* hist, unsign
         }
         const int above = incl - mine;
         const bool here = above < need && need <= incl;
-        int bin = 0, nd = 0;
+        int bin = 0, nd = 0, cb = 0;
         if (here) {
             int a = above;
             bin = lane * 8;
 #pragma unroll
             for (int b = 7; b >= 0; --b) {                 // highest bin whose suffix count reaches need
                 if (nd == 0) {
-                    if (a + c[b] >= need) { bin = lane * 8 + b; nd = need - a; }
+                    if (a + c[b] >= need) { bin = lane * 8 + b; nd = need - a; cb = c[b]; }
                     else a += c[b];
                 }
             }
@@ -56,9 +75,11 @@ __device__ void warp_radix_select(KeyFn keyf, int N, int need, int* hist, unsign
         const int src = __ffs(__ballot_sync(0xFFFFFFFFu, here)) - 1;
         bin = __shfl_sync(0xFFFFFFFFu, bin, src);
         need = __shfl_sync(0xFFFFFFFFu, nd, src);
-        prefix |= (unsigned long long)bin << (8 * pass);
-        pmask |= 0xFFull << (8 * pass);
+        cb = __shfl_sync(0xFFFFFFFFu, cb, src);
+        prefix |= (unsigned long long)bin << shift;
+        top = shift;
         __syncwarp();
+        if (cb == need && prefix != 0ull) { thr = prefix - 1ull; need_eq = 0; return; }   // the whole bin belongs
     }
     thr = prefix;
     need_eq = need;
@@ -85,6 +106,24 @@ __device__ int warp_compact_selected(KeyFn keyf, int N, unsigned long long thr, 
     return taken;
 }
 
+// The layer scratch of a CTA is shared by its finisher warps: a bounded spin lock in shared memory.
+__device__ __forceinline__ bool layer_lock(LayerScratch& s, int* status) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) {
+        const long long t0 = clock64();
+        while (atomicCAS(&s.lock, 0, 1) != 0) {
+            if (clock64() - t0 > kWaitCycles) { set_status(status, kErrTimeout); ok = 0; break; }
+            __nanosleep(100);
+        }
+        __threadfence_block();
+    }
+    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+}
+__device__ __forceinline__ void layer_unlock(LayerScratch& s) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) { __threadfence_block(); atomicExch(&s.lock, 0); }
+}
+
 // Per-sequence state and arrays in the workspace (device pointers already offset to the sequence).
 struct SeqWork {
     double* cand_phat;     // [n*k]    path values of this layer's candidates (Eq. 2), slot-major
@@ -94,7 +133,7 @@ struct SeqWork {
     double* T_phat;        // [D*n]
     int32_t* R;            // [2][n]   running top-n as gids in ascending order, double-buffered by layer parity
     double* E_prev;        // [1]      E of Algorithm 1
-    int32_t* st;           // [8]      0: frontier size, 1: rows finished in this layer, 2: |R|
+    int32_t* st;           // [8]      1: rows finished in this layer, 2: |R|
 };
 enum { kStFsize = 0, kStDone = 1, kStNR = 2 };
 
@@ -108,13 +147,14 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
 
 // After all rows of layer d (1-based) of one sequence are expanded: choose the layer, update the
 // running top-n and E_sub, apply the loop test, and pack the tree if the sequence is finished.
-// Whole finisher warp.  Returns the size of the new layer if the sequence continues with layer
-// d+1, or 0 if it is finished (outputs written).
-__device__ int finish_layer_warp(CtaSmem& s, const SeqWork& w, const TreeOut& out, int d, int n, int k, int kk,
-                                 int Dcap, int max_depth, float delta, int* status) {
+// Whole finisher warp; the caller holds the lock of the layer scratch s.  fsize = rows of the
+// layer.  Returns the size of the new layer if the sequence continues with layer d+1, or 0 if it
+// is finished (outputs written).
+__device__ int finish_layer_warp(LayerScratch& s, int* hist, const SeqWork& w, const TreeOut& out, int d, int fsize, int n, int k,
+                                 int kk, int Dcap, int max_depth, float delta, int* status) {
     const int lane = threadIdx.x & 31;
-    const int fsize = __ldcg(&w.st[kStFsize]);
-    const int nR_old = __ldcg(&w.st[kStNR]);
+    const int nR_old = d == 1 ? 0 : __ldcg(&w.st[kStNR]);
+    const double eprev = d == 1 ? 0.0 : __ldcg(w.E_prev);
     const int N = fsize * k;
     const int nvalid = fsize * kk;
     const int nl = nvalid < n ? nvalid : n;
@@ -123,21 +163,37 @@ __device__ int finish_layer_warp(CtaSmem& s, const SeqWork& w, const TreeOut& ou
     int need_eq;
 
     // --- next layer: the nl candidates of largest path value, stored in candidate-index order ---
-    auto emit_layer = [&](int pos, int i) {
-        w.T_tok[gid0 + pos] = __ldcg(&w.cand_tok[i]);
-        w.T_par[gid0 + pos] = i / k;
-        w.T_phat[gid0 + pos] = __ldcg(&w.cand_phat[i]);
-    };
     auto gkey = [&](int i) -> unsigned long long { return (i % k) < kk ? phat_key(__ldcg(&w.cand_phat[i])) : 0ull; };
-    if (N <= 1024) {                                      // stage the keys in shared memory
-        for (int i = lane; i < N; i += 32) s.keys[i] = gkey(i);
+    unsigned long long ko = 0ull, ka = ~0ull;
+    if (N <= 1024) {                                      // stage keys and tokens in shared memory
+        for (int i = lane; i < N; i += 32) {
+            const unsigned long long key = gkey(i);
+            s.keys[i] = key;
+            s.toks[i] = __ldcg(&w.cand_tok[i]);
+            if (key) { ko |= key; ka &= key; }
+        }
         __syncwarp();
         auto skey = [&](int i) -> unsigned long long { return s.keys[i]; };
-        warp_radix_select(skey, N, nl, s.hist, thr, need_eq);
-        warp_compact_selected(skey, N, thr, need_eq, emit_layer);
+        warp_radix_select(skey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
+        warp_compact_selected(skey, N, thr, need_eq, [&](int pos, int i) {
+            w.T_tok[gid0 + pos] = s.toks[i];
+            w.T_par[gid0 + pos] = i / k;
+            w.T_phat[gid0 + pos] = __longlong_as_double((long long)(s.keys[i] - 1ull));
+            s.lkeys[pos] = s.keys[i];
+        });
     } else {
-        warp_radix_select(gkey, N, nl, s.hist, thr, need_eq);
-        warp_compact_selected(gkey, N, thr, need_eq, emit_layer);
+        for (int i = lane; i < N; i += 32) {
+            const unsigned long long key = gkey(i);
+            if (key) { ko |= key; ka &= key; }
+        }
+        warp_radix_select(gkey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
+        warp_compact_selected(gkey, N, thr, need_eq, [&](int pos, int i) {
+            const unsigned long long key = gkey(i);
+            w.T_tok[gid0 + pos] = __ldcg(&w.cand_tok[i]);
+            w.T_par[gid0 + pos] = i / k;
+            w.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
+            s.lkeys[pos] = key;
+        });
     }
     __syncwarp();
 
@@ -146,27 +202,31 @@ __device__ int finish_layer_warp(CtaSmem& s, const SeqWork& w, const TreeOut& ou
     int32_t* Rnew = w.R + (d & 1) * n;
     const int NR = nR_old + nl;                           // <= 2n <= 512
     const int nR = NR < n ? NR : n;
+    ko = 0ull; ka = ~0ull;
     for (int i = lane; i < NR; i += 32) {
-        const int gid = i < nR_old ? __ldcg(&Rold[i]) : gid0 + (i - nR_old);
+        int gid;
+        unsigned long long key;
+        if (i < nR_old) { gid = __ldcg(&Rold[i]); key = phat_key(__ldcg(&w.T_phat[gid])); }
+        else { gid = gid0 + (i - nR_old); key = s.lkeys[i - nR_old]; }
         s.gids[i] = gid;
-        s.keys[i] = phat_key(__ldcg(&w.T_phat[gid]));
+        s.keys[i] = key;
+        ko |= key; ka &= key;
     }
     __syncwarp();
     auto rkey = [&](int i) -> unsigned long long { return s.keys[i]; };
-    warp_radix_select(rkey, NR, nR, s.hist, thr, need_eq);
+    warp_radix_select(rkey, NR, nR, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
     warp_compact_selected(rkey, NR, thr, need_eq, [&](int pos, int i) {
         Rnew[pos] = s.gids[i];
+        s.rsel[pos] = s.gids[i];
         s.vals[pos] = __longlong_as_double((long long)(s.keys[i] - 1ull));
     });
     __syncwarp();
     double part = 0.0;
     for (int i = lane; i < nR; i += 32) part += s.vals[i];
     const double esub = warp_sum(part);                   // fixed order: lanes stride the packed order
-    const double eprev = __ldcg(w.E_prev);
     const bool more = d < Dcap && (esub - eprev > (double)delta);     // loop test of Algorithm 1
     if (out.esub_trace && lane == 0) out.esub_trace[d - 1] = esub;
     if (lane == 0) {
-        w.st[kStFsize] = nl;
         w.st[kStNR] = nR;
         w.st[kStDone] = 0;
         *w.E_prev = esub;
@@ -179,7 +239,7 @@ __device__ int finish_layer_warp(CtaSmem& s, const SeqWork& w, const TreeOut& ou
         int32_t tok = -1, par = -1, dep = 0;
         double ph = 0.0;
         if (i < nR) {
-            const int gid = __ldcg(&Rnew[i]);
+            const int gid = s.rsel[i];
             dep = gid / n + 1;
             tok = __ldcg(&w.T_tok[gid]);
             ph = s.vals[i];
@@ -188,9 +248,9 @@ __device__ int finish_layer_warp(CtaSmem& s, const SeqWork& w, const TreeOut& ou
                 int lo = 0, hi = i;                        // the parent is packed before its child
                 while (lo < hi) {
                     const int mid = (lo + hi) >> 1;
-                    if (__ldcg(&Rnew[mid]) < pg) lo = mid + 1; else hi = mid;
+                    if (s.rsel[mid] < pg) lo = mid + 1; else hi = mid;
                 }
-                if (lo >= i || __ldcg(&Rnew[lo]) != pg) set_status(status, kErrInternal);   // closure violated
+                if (lo >= i || s.rsel[lo] != pg) set_status(status, kErrInternal);   // closure violated
                 par = lo;
             }
         }
