@@ -10,14 +10,16 @@ namespace ot {
 // CTA shape of the row pipeline (one CTA per SM): 16 consumer warps stream the logits, an issuer
 // warp feeds the shared-memory ring, a fetcher warp obtains row descriptors ahead of time, and
 // several finisher warps (one row each, round robin) turn finished rows into probabilities and
-// tree updates.  A lone warp advances slowly next to 16 busy ones, hence several finishers.
+// tree updates.  A lone warp advances slowly next to 16 busy ones, hence several finishers.  One
+// more warp takes whole-layer jobs of the tree build (selection of the next layer) from a queue.
 constexpr int kConsumerWarps = 16;
 constexpr int kConsumers = kConsumerWarps * 32;     // 512 consumer threads
 constexpr int kIssuerWarp = kConsumerWarps;         // warp 16
 constexpr int kFetcherWarp = kConsumerWarps + 1;    // warp 17
 constexpr int kFirstFinisherWarp = kConsumerWarps + 2;
 constexpr int kFinishers = 6;
-constexpr int kThreads = (kFirstFinisherWarp + kFinishers) * 32;   // 768 threads per CTA
+constexpr int kLayerWarp = kFirstFinisherWarp + kFinishers;
+constexpr int kThreads = (kLayerWarp + 1) * 32;     // 800 threads per CTA
 constexpr int kMaxK = 32;
 constexpr int kMaxN = 256;
 
@@ -165,6 +167,9 @@ __device__ __forceinline__ int ld_acquire_s32(const int* p) {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ void st_release_s32(int* p, int v) {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");

@@ -35,7 +35,9 @@ struct Workspace {
     int32_t* st;           // [B][8]
     // work queue of the build: one item per (sequence, layer, frontier slot)
     unsigned long long* q_items;   // [q_capacity]
-    int32_t* q_ctl;        // [8]  0: head (next to claim), 1: tail (published), 2: sequences finished, 3: all done
+    int32_t* q_ctl;        // [8]  0: head (next to claim), 1: tail (published), 2: sequences finished, 3: all done,
+                           //      4 / 5: head / tail of the layer-job queue
+    unsigned long long* lq_items;  // [lq_capacity]  one job per (sequence, layer) whose rows are all expanded
     // verify
     int32_t* g;            // [B][n+1]  target argmax after the root (0) and after node i (i+1)
     int32_t* vdone;        // [B]
@@ -47,7 +49,7 @@ struct Workspace {
     uint64_t* o_mask; int32_t* o_pos;
     int32_t *o_alen, *o_atok, *o_anode, *o_next;
 };
-enum { kQHead = 0, kQTail = 1, kQFinished = 2, kQDone = 3 };
+enum { kQHead = 0, kQTail = 1, kQFinished = 2, kQDone = 3, kLQHead = 4, kLQTail = 5 };
 
 constexpr int kQueueMargin = 4096;          // room for one over-claim per resident CTA
 
@@ -57,6 +59,11 @@ static size_t max_items(const opt_tree_config& c) {
     if (Dcap >= 2) per_seq += kk < n ? kk : n;
     if (Dcap >= 3) per_seq += (Dcap - 2) * n;
     return per_seq * (size_t)c.max_batch;
+}
+
+static size_t max_layer_jobs(const opt_tree_config& c) {
+    const size_t Dcap = c.max_depth < c.n ? c.max_depth : c.n;
+    return Dcap * (size_t)c.max_batch;
 }
 
 struct Layout {
@@ -83,6 +90,7 @@ static size_t carve(const opt_tree_config& c, char* base, Workspace* w) {
     OT_TAKE(st, int32_t, B * 8)
     OT_TAKE(q_items, unsigned long long, max_items(c) + kQueueMargin)
     OT_TAKE(q_ctl, int32_t, 8)
+    OT_TAKE(lq_items, unsigned long long, max_layer_jobs(c) + kQueueMargin)
     OT_TAKE(g, int32_t, B * (n + 1))
     OT_TAKE(vdone, int32_t, B)
     OT_TAKE(status, int32_t, 1)
@@ -109,7 +117,7 @@ struct Params {            // by-value kernel parameters
     int V, H, n, k, kk, Dcap, max_depth, B;
     float delta;
     int aligned;
-    int q_capacity;
+    int q_capacity, lq_capacity;
 };
 
 __device__ __forceinline__ SeqWork seq_work(const Workspace& w, const Params& p, int b) {
@@ -161,12 +169,16 @@ __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restri
         }
         w.q_items[i] = item;
     }
+    if (i < p.lq_capacity) w.lq_items[i] = 0ull;
     if (i < p.B) {
         int32_t* st = w.st + (size_t)i * 8;
         st[kStDone] = 0; st[kStNR] = 0;
         w.E_prev[i] = 0.0;
     }
-    if (i == 0) { w.q_ctl[kQHead] = 0; w.q_ctl[kQTail] = p.B; w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; }
+    if (i == 0) {
+        w.q_ctl[kQHead] = 0; w.q_ctl[kQTail] = p.B; w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0;
+        w.q_ctl[kLQHead] = 0; w.q_ctl[kLQTail] = 0;
+    }
 }
 
 // Source of the tree build: rows come from the global work queue.
@@ -196,11 +208,17 @@ struct BuildSource {
     }
 };
 
-// Sink of the tree build: candidates' path values (Eq. 2), then, for the row that completes its
-// layer, the layer selection / loop test, and either new queue items or the packed tree.
+// Layer job: bit 63 valid | b (15 bits) | layer d (9) | rows in the layer (9).
+__device__ __forceinline__ unsigned long long job_encode(int b, int d, int fsize) {
+    return (1ull << 63) | ((unsigned long long)b << 48) | ((unsigned long long)d << 39) | ((unsigned long long)fsize << 30);
+}
+
+// Sink of the tree build.  Finisher warps: candidates' path values (Eq. 2); the row that completes
+// its layer posts a layer job.  Layer warp: takes jobs, does the layer selection / loop test, and
+// either publishes the next layer's rows or leaves the packed tree.
 struct BuildSink {
-    CtaSmem* s; Workspace w; Params p; opt_tree_out out;
-    __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch& f) {
+    Workspace w; Params p; opt_tree_out out;
+    __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch&) {
         const int lane = threadIdx.x & 31;
         const SeqWork sw = seq_work(w, p, d.b);
         const double parent_phat = d.d == 1 ? 1.0 : __ldcg(&sw.T_phat[(size_t)(d.d - 2) * p.n + d.slot]);   // root: factor 1
@@ -210,29 +228,52 @@ struct BuildSink {
         }
         __threadfence();
         __syncwarp();
-        int last = 0;
-        if (lane == 0) last = atomicAdd(&sw.st[kStDone], 1) == d.fsize - 1;
-        last = __shfl_sync(0xFFFFFFFFu, last, 0);
-        if (!last) return;
-        __threadfence();
-        if (!layer_lock(s->layer, w.status)) return;
-        const int nl = finish_layer_warp(s->layer, f.hist, sw, tree_out(out, p, d.b), d.d, d.fsize, p.n, p.k, p.kk, p.Dcap,
-                                         p.max_depth, p.delta, w.status);
-        layer_unlock(s->layer);
-        __threadfence();
-        __syncwarp();
-        if (nl > 0) {
-            int pos = 0;
-            if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
-            pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
-            for (int i = lane; i < nl; i += 32) {
-                int token = __ldcg(&sw.T_tok[(size_t)(d.d - 1) * p.n + i]);
-                if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
-                if (pos + i < p.q_capacity) st_release_u64(&w.q_items[pos + i], item_encode(d.b, d.d + 1, nl, i, row_of(token, d.d, p.H)));
-                else set_status(w.status, kErrInternal);
+        if (lane == 0 && atomicAdd(&sw.st[kStDone], 1) == d.fsize - 1) {
+            __threadfence();
+            const int pos = atomicAdd(&w.q_ctl[kLQTail], 1);
+            if (pos < p.lq_capacity) st_release_u64(&w.lq_items[pos], job_encode(d.b, d.d, d.fsize));
+            else set_status(w.status, kErrInternal);
+        }
+    }
+    __device__ void layer_loop(LayerScratch& ls) {
+        const int lane = threadIdx.x & 31;
+        for (;;) {
+            unsigned long long job = 0ull;
+            if (lane == 0) {
+                const int idx = atomicAdd(&w.q_ctl[kLQHead], 1);
+                if (idx < p.lq_capacity) {
+                    const long long t0 = clock64();
+                    for (;;) {
+                        job = ld_acquire_u64(&w.lq_items[idx]);
+                        if (job >> 63) break;
+                        if (ld_acquire_s32(&w.q_ctl[kQDone])) { job = 0ull; break; }
+                        if (clock64() - t0 > kWaitCycles) { set_status(w.status, kErrTimeout); job = 0ull; break; }
+                        __nanosleep(200);
+                    }
+                }
             }
-        } else if (lane == 0) {
-            if (atomicAdd(&w.q_ctl[kQFinished], 1) == p.B - 1) st_release_s32(&w.q_ctl[kQDone], 1);
+            job = __shfl_sync(0xFFFFFFFFu, job, 0);
+            if (!(job >> 63)) return;
+            const int b = (int)((job >> 48) & 0x7FFFu), d = (int)((job >> 39) & 0x1FFu), fsize = (int)((job >> 30) & 0x1FFu);
+            const SeqWork sw = seq_work(w, p, b);
+            const int nl = finish_layer_warp(ls, sw, tree_out(out, p, b), d, fsize, p.n, p.k, p.kk, p.Dcap, p.max_depth, p.delta, w.status);
+            __syncwarp();
+            if (nl > 0) {
+                int pos = 0;
+                if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
+                pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
+                __threadfence();                               // the layer's nodes before its queue items
+                for (int i = lane; i < nl; i += 32) {
+                    int token = ls.ltok[i];
+                    if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
+                    if (pos + i < p.q_capacity) st_relaxed_u64(&w.q_items[pos + i], item_encode(b, d + 1, nl, i, row_of(token, d, p.H)));
+                    else set_status(w.status, kErrInternal);
+                }
+            } else {
+                __threadfence();
+                if (lane == 0 && atomicAdd(&w.q_ctl[kQFinished], 1) == p.B - 1) st_release_s32(&w.q_ctl[kQDone], 1);
+            }
+            __syncwarp();
         }
     }
 };
@@ -244,7 +285,7 @@ build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, opt_tree
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
     BuildSource src{w, p, draft};
-    BuildSink sink{&s, w, p, out};
+    BuildSink sink{w, p, out};
     run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, w.status);
 }
 
@@ -262,6 +303,7 @@ struct ListSource {
 };
 struct ListSink {
     int32_t* tok_out; double* prob_out; int k;
+    __device__ void layer_loop(LayerScratch&) {}
     __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch&) {
         const int lane = threadIdx.x & 31;
         if (lane < k) {
@@ -433,7 +475,7 @@ struct opt_tree_ctx {
     size_t bytes;
     int device;
     int grid;              // resident CTAs of the persistent kernels (SMs x occupancy)
-    int q_capacity;
+    int q_capacity, lq_capacity;
     int64_t launches;
 };
 
@@ -456,6 +498,7 @@ ot::Params make_params(const opt_tree_ctx* ctx, const void* table, float delta) 
     p.max_depth = c.max_depth;
     p.B = 0;
     p.q_capacity = ctx->q_capacity;
+    p.lq_capacity = ctx->lq_capacity;
     p.delta = delta;
     p.aligned = ((reinterpret_cast<uintptr_t>(table) & 15u) == 0 && (c.V % 8) == 0) ? 1 : 0;
     return p;
@@ -492,6 +535,7 @@ int opt_tree_create(opt_tree_ctx** out, const opt_tree_config* cfg) {
     }
     ot::carve(*cfg, static_cast<char*>(ctx->base), &ctx->ws);
     ctx->q_capacity = (int)(ot::max_items(*cfg) + ot::kQueueMargin);
+    ctx->lq_capacity = (int)(ot::max_layer_jobs(*cfg) + ot::kQueueMargin);
     bool ok = cudaMemset(ctx->base, 0, ctx->bytes) == cudaSuccess;
     ok = ok && cudaFuncSetAttribute(ot::build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)sizeof(ot::CtaSmem)) == cudaSuccess;
@@ -526,7 +570,7 @@ int opt_tree_build(opt_tree_ctx* ctx, const void* draft, const int32_t* root_tok
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     ot::Params p = make_params(ctx, draft, delta);
     p.B = B;
-    ot::init_build_kernel<<<(ctx->q_capacity + 255) / 256, 256, 0, st>>>(ctx->ws, p, root_token);
+    ot::init_build_kernel<<<((ctx->q_capacity > ctx->lq_capacity ? ctx->q_capacity : ctx->lq_capacity) + 255) / 256, 256, 0, st>>>(ctx->ws, p, root_token);
     ot::build_kernel<<<ctx->grid, ot::kThreads, sizeof(ot::CtaSmem), st>>>(
         ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
     ctx->launches += 2;

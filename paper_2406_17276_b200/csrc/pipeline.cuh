@@ -8,8 +8,10 @@
 //                   per-thread maxima and partial sums to a finisher through a slot and go
 //                   straight on to the next row;
 //   finisher warps  row r goes to finisher r mod kFinishers: it computes the row's winners and
-//                   gives them to a Sink (which may, for the tree build, select a layer and
-//                   publish new rows).
+//                   gives them to a Sink (for the tree build: candidates' path values, and a
+//                   layer job once a layer's last row is in);
+//   layer warp      runs Sink::layer_loop (for the tree build: takes layer jobs from a queue,
+//                   selects the next layer and publishes its rows).
 //
 // The chunks of consecutive rows form one stream: chunk g lives in stage g % kStages and is the
 // (g / kStages)-th use of that stage, which fixes every mbarrier parity; likewise row r uses
@@ -28,7 +30,6 @@ __device__ __forceinline__ void pipeline_init(CtaSmem& s) {
         for (int i = 0; i < kSlots; ++i) { mbar_init(&s.ready_bar[i], kConsumerWarps); mbar_init(&s.free_bar[i], 1); }
         for (int i = 0; i < kDesc; ++i) { mbar_init(&s.desc_full[i], 1); mbar_init(&s.desc_empty[i], kConsumerWarps); }
         s.stop_row = 0x7FFFFFFF;
-        s.layer.lock = 0;
         mbar_fence_init();
     }
     __syncthreads();
@@ -171,6 +172,7 @@ __device__ __forceinline__ void run_pipeline(CtaSmem& s, Source& src, Sink& sink
     if (warp < kConsumerWarps) consumer_role(s, V, status);
     else if (warp == kIssuerWarp) issuer_role(s, V, aligned, status);
     else if (warp == kFetcherWarp) fetcher_role(s, src, status);
+    else if (warp == kLayerWarp) sink.layer_loop(s.layer);
     else finisher_role(s, sink, warp - kFirstFinisherWarp, V, k, aligned, status);
 }
 

@@ -66,14 +66,15 @@ struct FinScratch {                // private to one finisher warp
     int cand_count;
 };
 
-struct LayerScratch {              // shared by the finisher warps of a CTA under `lock`
+struct LayerScratch {              // private to the layer warp of a CTA
     unsigned long long keys[1024];             // staged candidate keys, then the keys of R + layer
     unsigned long long lkeys[kMaxN];           // keys of the new layer, slot order
     double vals[kMaxN];                        // path values of the new running top-n
     int toks[1024];                            // staged candidate tokens
     int gids[2 * kMaxN];
     int rsel[kMaxN];                           // gids of the new running top-n, ascending
-    int lock;
+    int ltok[kMaxN];                           // tokens of the new layer, slot order
+    int hist[256];
 };
 
 struct alignas(128) CtaSmem {

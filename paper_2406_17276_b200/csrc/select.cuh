@@ -106,24 +106,6 @@ __device__ int warp_compact_selected(KeyFn keyf, int N, unsigned long long thr, 
     return taken;
 }
 
-// The layer scratch of a CTA is shared by its finisher warps: a bounded spin lock in shared memory.
-__device__ __forceinline__ bool layer_lock(LayerScratch& s, int* status) {
-    int ok = 1;
-    if ((threadIdx.x & 31) == 0) {
-        const long long t0 = clock64();
-        while (atomicCAS(&s.lock, 0, 1) != 0) {
-            if (clock64() - t0 > kWaitCycles) { set_status(status, kErrTimeout); ok = 0; break; }
-            __nanosleep(100);
-        }
-        __threadfence_block();
-    }
-    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
-}
-__device__ __forceinline__ void layer_unlock(LayerScratch& s) {
-    __syncwarp();
-    if ((threadIdx.x & 31) == 0) { __threadfence_block(); atomicExch(&s.lock, 0); }
-}
-
 // Per-sequence state and arrays in the workspace (device pointers already offset to the sequence).
 struct SeqWork {
     double* cand_phat;     // [n*k]    path values of this layer's candidates (Eq. 2), slot-major
@@ -147,12 +129,12 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
 
 // After all rows of layer d (1-based) of one sequence are expanded: choose the layer, update the
 // running top-n and E_sub, apply the loop test, and pack the tree if the sequence is finished.
-// Whole finisher warp; the caller holds the lock of the layer scratch s.  fsize = rows of the
-// layer.  Returns the size of the new layer if the sequence continues with layer d+1, or 0 if it
+// Whole layer warp; s is its scratch.  fsize = rows of the layer.  Returns the size of the new layer if the sequence continues with layer d+1, or 0 if it
 // is finished (outputs written).
-__device__ int finish_layer_warp(LayerScratch& s, int* hist, const SeqWork& w, const TreeOut& out, int d, int fsize, int n, int k,
+__device__ int finish_layer_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int fsize, int n, int k,
                                  int kk, int Dcap, int max_depth, float delta, int* status) {
     const int lane = threadIdx.x & 31;
+    int* hist = s.hist;
     const int nR_old = d == 1 ? 0 : __ldcg(&w.st[kStNR]);
     const double eprev = d == 1 ? 0.0 : __ldcg(w.E_prev);
     const int N = fsize * k;
@@ -177,6 +159,7 @@ __device__ int finish_layer_warp(LayerScratch& s, int* hist, const SeqWork& w, c
         warp_radix_select(skey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
         warp_compact_selected(skey, N, thr, need_eq, [&](int pos, int i) {
             w.T_tok[gid0 + pos] = s.toks[i];
+            s.ltok[pos] = s.toks[i];
             w.T_par[gid0 + pos] = i / k;
             w.T_phat[gid0 + pos] = __longlong_as_double((long long)(s.keys[i] - 1ull));
             s.lkeys[pos] = s.keys[i];
@@ -189,7 +172,9 @@ __device__ int finish_layer_warp(LayerScratch& s, int* hist, const SeqWork& w, c
         warp_radix_select(gkey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
         warp_compact_selected(gkey, N, thr, need_eq, [&](int pos, int i) {
             const unsigned long long key = gkey(i);
-            w.T_tok[gid0 + pos] = __ldcg(&w.cand_tok[i]);
+            const int tok = __ldcg(&w.cand_tok[i]);
+            w.T_tok[gid0 + pos] = tok;
+            s.ltok[pos] = tok;
             w.T_par[gid0 + pos] = i / k;
             w.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
             s.lkeys[pos] = key;
