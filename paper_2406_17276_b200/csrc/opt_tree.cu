@@ -172,7 +172,7 @@ __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restri
     if (i < p.lq_capacity) w.lq_items[i] = 0ull;
     if (i < p.B) {
         int32_t* st = w.st + (size_t)i * 8;
-        st[kStDone] = 0; st[kStNR] = 0;
+        st[kStDone] = 0; st[kStNR] = 0; st[kStUpdated] = 0;
         w.E_prev[i] = 0.0;
     }
     if (i == 0) {
@@ -235,6 +235,21 @@ struct BuildSink {
             else set_status(w.status, kErrInternal);
         }
     }
+    // Queue items for the rows of layer d+1 (the nodes select_layer_warp just chose).
+    __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl) {
+        const int lane = threadIdx.x & 31;
+        int pos = 0;
+        if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
+        pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
+        __threadfence();                                   // the layer's nodes before its queue items
+        for (int i = lane; i < nl; i += 32) {
+            int token = ls.ltok[i];
+            if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
+            if (pos + i < p.q_capacity) st_relaxed_u64(&w.q_items[pos + i], item_encode(b, d + 1, nl, i, row_of(token, d, p.H)));
+            else set_status(w.status, kErrInternal);
+        }
+        __syncwarp();
+    }
     __device__ void layer_loop(LayerScratch& ls) {
         const int lane = threadIdx.x & 31;
         for (;;) {
@@ -256,20 +271,14 @@ struct BuildSink {
             if (!(job >> 63)) return;
             const int b = (int)((job >> 48) & 0x7FFFu), d = (int)((job >> 39) & 0x1FFu), fsize = (int)((job >> 30) & 0x1FFu);
             const SeqWork sw = seq_work(w, p, b);
-            const int nl = finish_layer_warp(ls, sw, tree_out(out, p, b), d, fsize, p.n, p.k, p.kk, p.Dcap, p.max_depth, p.delta, w.status);
-            __syncwarp();
-            if (nl > 0) {
-                int pos = 0;
-                if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
-                pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
-                __threadfence();                               // the layer's nodes before its queue items
-                for (int i = lane; i < nl; i += 32) {
-                    int token = ls.ltok[i];
-                    if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
-                    if (pos + i < p.q_capacity) st_relaxed_u64(&w.q_items[pos + i], item_encode(b, d + 1, nl, i, row_of(token, d, p.H)));
-                    else set_status(w.status, kErrInternal);
-                }
-            } else {
+            const int nl = select_layer_warp(ls, sw, d, fsize, p.n, p.k, p.kk);
+            // Without a threshold the loop test only looks at the depth: the next layer's rows can
+            // go out before the running top-n is brought up to date.
+            const bool early = d < p.Dcap && p.delta == -INFINITY;
+            if (early) publish_layer(ls, b, d, nl);
+            const bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta, w.status);
+            if (more && !early) publish_layer(ls, b, d, nl);
+            if (!more && !early) {
                 __threadfence();
                 if (lane == 0 && atomicAdd(&w.q_ctl[kQFinished], 1) == p.B - 1) st_release_s32(&w.q_ctl[kQDone], 1);
             }

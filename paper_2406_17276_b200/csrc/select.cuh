@@ -115,9 +115,9 @@ struct SeqWork {
     double* T_phat;        // [D*n]
     int32_t* R;            // [2][n]   running top-n as gids in ascending order, double-buffered by layer parity
     double* E_prev;        // [1]      E of Algorithm 1
-    int32_t* st;           // [8]      1: rows finished in this layer, 2: |R|
+    int32_t* st;           // [8]      1: rows finished in this layer, 2: |R|, 3: last layer folded into R
 };
-enum { kStFsize = 0, kStDone = 1, kStNR = 2 };
+enum { kStDone = 1, kStNR = 2, kStUpdated = 3 };
 
 struct TreeOut {           // mirrors opt_tree_out, pointers offset to the sequence
     int32_t *token, *parent, *depth;
@@ -127,27 +127,23 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
     double* esub_trace;    // may be null
 };
 
-// After all rows of layer d (1-based) of one sequence are expanded: choose the layer, update the
-// running top-n and E_sub, apply the loop test, and pack the tree if the sequence is finished.
-// Whole layer warp; s is its scratch.  fsize = rows of the layer.  Returns the size of the new layer if the sequence continues with layer d+1, or 0 if it
-// is finished (outputs written).
-__device__ int finish_layer_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int fsize, int n, int k,
-                                 int kk, int Dcap, int max_depth, float delta, int* status) {
+// Layer job, first half.  After all rows of layer d (1-based) of one sequence are expanded: the
+// next layer = the nl candidates of largest path value, stored in candidate-index order (nodes
+// gid0 .. gid0+nl of T; tokens and keys also left in s.ltok / s.lkeys).  Resets the sequence's
+// row counter.  Whole layer warp; s is its scratch; fsize = rows of the layer.  Returns nl.
+__device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int fsize, int n, int k, int kk) {
     const int lane = threadIdx.x & 31;
     int* hist = s.hist;
-    const int nR_old = d == 1 ? 0 : __ldcg(&w.st[kStNR]);
-    const double eprev = d == 1 ? 0.0 : __ldcg(w.E_prev);
     const int N = fsize * k;
     const int nvalid = fsize * kk;
     const int nl = nvalid < n ? nvalid : n;
     const int gid0 = (d - 1) * n;
     unsigned long long thr;
     int need_eq;
-
-    // --- next layer: the nl candidates of largest path value, stored in candidate-index order ---
     auto gkey = [&](int i) -> unsigned long long { return (i % k) < kk ? phat_key(__ldcg(&w.cand_phat[i])) : 0ull; };
     unsigned long long ko = 0ull, ka = ~0ull;
     if (N <= 1024) {                                      // stage keys and tokens in shared memory
+#pragma unroll 4
         for (int i = lane; i < N; i += 32) {
             const unsigned long long key = gkey(i);
             s.keys[i] = key;
@@ -180,14 +176,44 @@ __device__ int finish_layer_warp(LayerScratch& s, const SeqWork& w, const TreeOu
             s.lkeys[pos] = key;
         });
     }
+    if (lane == 0) w.st[kStDone] = 0;
     __syncwarp();
+    return nl;
+}
+
+// Layer job, second half: the running top-n and E_sub(T, n) with the new layer (left in s by
+// select_layer_warp), the loop test of Algorithm 1, and the packed tree if the sequence is
+// finished.  Layer d's update must follow layer d-1's (they may run on different CTAs): the
+// sequence's st[kStUpdated] holds the last layer whose update is complete.  Returns true if the
+// sequence continues with layer d+1, false if it is finished (outputs written) or a wait expired.
+__device__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
+                                    int max_depth, float delta, int* status) {
+    const int lane = threadIdx.x & 31;
+    int* hist = s.hist;
+    const int gid0 = (d - 1) * n;
+    unsigned long long thr;
+    int need_eq;
+    if (d > 1) {
+        int ok = 1;
+        if (lane == 0) {
+            const long long t0 = clock64();
+            while (ld_acquire_s32(&w.st[kStUpdated]) < d - 1) {
+                if (clock64() - t0 > kWaitCycles) { set_status(status, kErrTimeout); ok = 0; break; }
+                __nanosleep(100);
+            }
+        }
+        if (!__shfl_sync(0xFFFFFFFFu, ok, 0)) return false;
+    }
+    const int nR_old = d == 1 ? 0 : __ldcg(&w.st[kStNR]);
+    const double eprev = d == 1 ? 0.0 : __ldcg(w.E_prev);
 
     // --- E_sub(T, n): the n largest path values among the previous top-n and the new layer ---
     const int32_t* Rold = w.R + ((d - 1) & 1) * n;
     int32_t* Rnew = w.R + (d & 1) * n;
     const int NR = nR_old + nl;                           // <= 2n <= 512
     const int nR = NR < n ? NR : n;
-    ko = 0ull; ka = ~0ull;
+    unsigned long long ko = 0ull, ka = ~0ull;
+#pragma unroll 4
     for (int i = lane; i < NR; i += 32) {
         int gid;
         unsigned long long key;
@@ -213,10 +239,12 @@ __device__ int finish_layer_warp(LayerScratch& s, const SeqWork& w, const TreeOu
     if (out.esub_trace && lane == 0) out.esub_trace[d - 1] = esub;
     if (lane == 0) {
         w.st[kStNR] = nR;
-        w.st[kStDone] = 0;
         *w.E_prev = esub;
     }
-    if (more) return nl;
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) st_release_s32(&w.st[kStUpdated], d);
+    if (more) return true;
 
     // --- pack: T_opt = the running top-n, already in (depth, parent's index, sibling rank) order ---
     if (out.esub_trace) for (int i = d + lane; i < max_depth; i += 32) out.esub_trace[i] = 0.0;
@@ -242,7 +270,7 @@ __device__ int finish_layer_warp(LayerScratch& s, const SeqWork& w, const TreeOu
         out.token[i] = tok; out.parent[i] = par; out.depth[i] = dep; out.phat[i] = ph;
     }
     if (lane == 0) { *out.n_sel = nR; *out.depth_reached = d; *out.expected_len = esub; }
-    return 0;
+    return false;
 }
 
 }  // namespace ot
