@@ -118,6 +118,34 @@ int opt_tree_verify(opt_tree_ctx *ctx, const opt_tree_out *tree, const void *tar
                     const int32_t *root_token, int32_t B, int32_t *accept_len, int32_t *accept_tokens,
                     int32_t *accept_nodes, int32_t *next_root, void *stream);
 
+/* Greedy verification for callers that must not allocate (the paper has no counterpart; this is a
+ * packaging variant of opt_tree_verify, same kernel, same results).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a serving engine that owns
+ * the whole device heap through its own pool and forbids driver allocations after start-up, or in a
+ * latency-critical loop where an allocation's implicit device synchronisation is unacceptable.  Such
+ * a caller cannot make an opt_tree_ctx (opt_tree_create allocates the workspace), so this entry
+ * point takes the problem sizes directly and keeps the kernel's scratch (the target's best token
+ * per node, one arrival counter per sequence, a status word) in a fixed array that is part of the
+ * library image: about 65 KB on every GPU that loads the library, held until the process exits.
+ *
+ * Limits: B <= OPT_TREE_STATIC_MAX_BATCH and cfg->n <= OPT_TREE_STATIC_MAX_N, otherwise
+ * OPT_TREE_ERR_UNSUPPORTED and nothing is launched.  cfg->max_batch is ignored.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine; it enqueues one small
+ * memset, the kernel and (if device_status is given) one 4-byte device-to-device copy on `stream`.
+ * The first call on each device asks the runtime for the array's device address (with that device
+ * current); make that first call outside any stream capture.
+ * Every call on a device shares the one array: two calls whose kernels may overlap on the GPU
+ * (different streams, no dependency between them) race on it -- order them.  The array keeps what
+ * the last call wrote; each call clears the counters and the status word before its kernel.
+ *   tree, target_logits_bf16, root_token, accept_*, next_root: as for opt_tree_verify
+ *   device_status (dev) [1] or NULL: receives OPT_TREE_OK or the first device-side error of this call */
+#define OPT_TREE_STATIC_MAX_BATCH 64
+#define OPT_TREE_STATIC_MAX_N 256
+int opt_tree_verify_static(const opt_tree_config *cfg, const opt_tree_out *tree, const void *target_logits_bf16,
+                           const int32_t *root_token, int32_t B, int32_t *accept_len, int32_t *accept_tokens,
+                           int32_t *accept_nodes, int32_t *next_root, int32_t *device_status, void *stream);
+
 /* The row step of Algorithm 1 on its own (children rule after Eq. 2): for each listed row,
  * the min(k, V) most probable tokens (logit descending, token id ascending) and their softmax
  * probabilities.

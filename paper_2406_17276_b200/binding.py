@@ -19,7 +19,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -
 
 EXPORTS = ["opt_tree_workspace_bytes", "opt_tree_create", "opt_tree_destroy", "opt_tree_build", "opt_tree_mask",
            "opt_tree_verify", "opt_tree_row_softmax_topk", "opt_tree_step_host", "opt_tree_last_device_status",
-           "opt_tree_launch_count", "opt_tree_strerror"]
+           "opt_tree_launch_count", "opt_tree_strerror", "opt_tree_verify_static"]
 
 
 class Config(C.Structure):
@@ -63,6 +63,8 @@ def lib():
         L.opt_tree_last_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
         L.opt_tree_launch_count.restype = C.c_int64
         L.opt_tree_launch_count.argtypes = [C.c_void_p]
+        L.opt_tree_verify_static.argtypes = [C.POINTER(Config), C.POINTER(Out), C.c_void_p, C.c_void_p, C.c_int32,
+                                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.opt_tree_strerror.restype = C.c_char_p
         L.opt_tree_strerror.argtypes = [C.c_int]
         _lib = L
@@ -206,3 +208,13 @@ class OptTree:
 
     def launch_count(self) -> int:
         return int(lib().opt_tree_launch_count(self._ctx))
+
+
+def verify_static(cfg: Config, tree: Tree, target: torch.Tensor, root_token: torch.Tensor, out, device_status: torch.Tensor | None = None):
+    """opt_tree_verify_static: verification for callers that cannot allocate.  Needs no OptTree context; every
+    buffer, outputs included, is the caller's (out = (accept_len, accept_tokens, accept_nodes, next_root))."""
+    B = tree.token.shape[0]
+    cs = tree.c_struct()
+    _check(lib().opt_tree_verify_static(C.byref(cfg), C.byref(cs), _ptr(target), _ptr(root_token), B, _ptr(out[0]), _ptr(out[1]),
+                                        _ptr(out[2]), _ptr(out[3]), _ptr(device_status), _stream()), "opt_tree_verify_static")
+    return out

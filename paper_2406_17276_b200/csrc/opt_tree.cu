@@ -667,3 +667,72 @@ const char* opt_tree_strerror(int code) {
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Verification without any allocation (opt_tree_verify_static).
+// ------------------------------------------------------------------------------------------------
+// The verify kernel needs three pieces of scratch: the target's best token per node, a per-sequence
+// arrival counter and a status word.  A context keeps them in memory it got from cudaMalloc; this
+// variant keeps them in the array below, which is part of the loaded library image on every GPU.
+namespace {
+
+constexpr size_t kStaticG = (size_t)OPT_TREE_STATIC_MAX_BATCH * (OPT_TREE_STATIC_MAX_N + 1);   // ints
+constexpr size_t kStaticInts = kStaticG + OPT_TREE_STATIC_MAX_BATCH + 1;
+constexpr size_t kStaticBytes = (kStaticInts * sizeof(int32_t) + 255) & ~(size_t)255;
+
+static __device__ __align__(256) unsigned char g_verify_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+int32_t* g_scratch_addr[kMaxDevices];      // device address of g_verify_scratch on each device, once looked up
+
+// The array's name means nothing to a kernel when used from host code; the device address comes from
+// the runtime, once per device, with that device current.  No lock: two threads racing here both
+// store the same value.
+int static_scratch(int32_t** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return OPT_TREE_ERR_CUDA;
+    if (!g_scratch_addr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_verify_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return OPT_TREE_ERR_CUDA;
+        }
+        g_scratch_addr[dev] = static_cast<int32_t*>(ptr);
+    }
+    *out = g_scratch_addr[dev];
+    return OPT_TREE_OK;
+}
+
+}  // namespace
+
+extern "C" int opt_tree_verify_static(const opt_tree_config* cfg, const opt_tree_out* tree, const void* target,
+                                      const int32_t* root_token, int32_t B, int32_t* accept_len, int32_t* accept_tokens,
+                                      int32_t* accept_nodes, int32_t* next_root, int32_t* device_status, void* stream) {
+    if (!valid_cfg(cfg) || bad_tree(tree) || !target || !root_token || !accept_len || !accept_tokens || !accept_nodes ||
+        !next_root || B < 1)
+        return OPT_TREE_ERR_INVALID_ARG;
+    if (supported_cfg(cfg) != OPT_TREE_OK) return OPT_TREE_ERR_UNSUPPORTED;
+    if (B > OPT_TREE_STATIC_MAX_BATCH || cfg->n > OPT_TREE_STATIC_MAX_N) return OPT_TREE_ERR_UNSUPPORTED;
+    int32_t* base = nullptr;
+    const int rc = static_scratch(&base);
+    if (rc != OPT_TREE_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ot::Workspace ws;
+    memset(&ws, 0, sizeof ws);
+    ws.g = base;
+    ws.vdone = base + kStaticG;
+    ws.status = base + kStaticG + OPT_TREE_STATIC_MAX_BATCH;
+    // counters and status start from zero whatever the previous call left behind
+    if (cudaMemsetAsync(ws.vdone, 0, (OPT_TREE_STATIC_MAX_BATCH + 1) * sizeof(int32_t), st) != cudaSuccess) return OPT_TREE_ERR_CUDA;
+    ot::Params p;
+    memset(&p, 0, sizeof p);
+    p.V = cfg->V; p.H = cfg->H; p.n = cfg->n; p.k = cfg->k; p.kk = cfg->k < cfg->V ? cfg->k : cfg->V;
+    p.max_depth = cfg->max_depth; p.Dcap = cfg->max_depth < cfg->n ? cfg->max_depth : cfg->n;
+    p.aligned = ((reinterpret_cast<uintptr_t>(target) & 15u) == 0 && (cfg->V % 8) == 0) ? 1 : 0;
+    ot::verify_kernel<<<dim3(cfg->n + 1, B), ot::kSmallThreads, 0, st>>>(
+        ws, p, static_cast<const uint16_t*>(target), root_token, *tree, accept_len, accept_tokens, accept_nodes, next_root);
+    if (cudaGetLastError() != cudaSuccess) return OPT_TREE_ERR_CUDA;
+    if (device_status && cudaMemcpyAsync(device_status, ws.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return OPT_TREE_ERR_CUDA;
+    return OPT_TREE_OK;
+}
