@@ -213,7 +213,7 @@ def run_cuda(args):
         "e2e": {"value": world * B / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "opt_tree_build (init + one build_round_kernel per layer)",
+        "roofline": {"bound": "hbm", "kernel": "build_kernel (opt_tree_build: init_build_kernel + one persistent build_kernel)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / 8000.0,
                      "algorithmic_bytes_per_build_call": algo_bytes, "build_ms": build_ms, "traffic": args.traffic},
