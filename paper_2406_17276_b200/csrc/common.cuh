@@ -154,11 +154,43 @@ __device__ __forceinline__ bool mbar_wait_warp(unsigned long long* bar, uint32_t
     return __all_sync(0xFFFFFFFFu, ok);
 }
 
+// Non-blocking test of a phase (does not suspend the thread).
+__device__ __forceinline__ bool mbar_test_wait(unsigned long long* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// The same wait for a single thread whose warp mates are busy elsewhere (no warp-wide vote).
+__device__ __forceinline__ bool mbar_wait_thread(unsigned long long* bar, uint32_t parity, int* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    long long t0 = 0;
+    int turns = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++turns & 255) == 0) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitCycles) { set_status(status, kErrTimeout); return false; }
+        }
+    }
+    return true;
+}
+
 // --- global-memory flags and queue words (gpu scope) ---
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
     unsigned long long v;
     asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void atom_add_release_s32(int* p, int v) {
+    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
     asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");

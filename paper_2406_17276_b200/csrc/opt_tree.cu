@@ -35,9 +35,8 @@ struct Workspace {
     int32_t* st;           // [B][8]
     // work queue of the build: one item per (sequence, layer, frontier slot)
     unsigned long long* q_items;   // [q_capacity]
-    int32_t* q_ctl;        // [8]  0: head (next to claim), 1: tail (published), 2: sequences finished, 3: all done,
-                           //      4 / 5: head / tail of the layer-job queue
-    unsigned long long* lq_items;  // [lq_capacity]  one job per (sequence, layer) whose rows are all expanded
+    unsigned long long* q_phat;    // [q_capacity]  bit 63 valid | bits of the parent's path value (a double >= 0)
+    int32_t* q_ctl;        // [8]  0: head (next to claim), 1: tail (published), 2: sequences finished, 3: all done
     // verify
     int32_t* g;            // [B][n+1]  target argmax after the root (0) and after node i (i+1)
     int32_t* vdone;        // [B]
@@ -49,7 +48,7 @@ struct Workspace {
     uint64_t* o_mask; int32_t* o_pos;
     int32_t *o_alen, *o_atok, *o_anode, *o_next;
 };
-enum { kQHead = 0, kQTail = 1, kQFinished = 2, kQDone = 3, kLQHead = 4, kLQTail = 5 };
+enum { kQHead = 0, kQTail = 1, kQFinished = 2, kQDone = 3 };
 
 constexpr int kQueueMargin = 4096;          // room for one over-claim per resident CTA
 
@@ -59,11 +58,6 @@ static size_t max_items(const opt_tree_config& c) {
     if (Dcap >= 2) per_seq += kk < n ? kk : n;
     if (Dcap >= 3) per_seq += (Dcap - 2) * n;
     return per_seq * (size_t)c.max_batch;
-}
-
-static size_t max_layer_jobs(const opt_tree_config& c) {
-    const size_t Dcap = c.max_depth < c.n ? c.max_depth : c.n;
-    return Dcap * (size_t)c.max_batch;
 }
 
 struct Layout {
@@ -89,8 +83,8 @@ static size_t carve(const opt_tree_config& c, char* base, Workspace* w) {
     OT_TAKE(E_prev, double, B)
     OT_TAKE(st, int32_t, B * 8)
     OT_TAKE(q_items, unsigned long long, max_items(c) + kQueueMargin)
+    OT_TAKE(q_phat, unsigned long long, max_items(c) + kQueueMargin)
     OT_TAKE(q_ctl, int32_t, 8)
-    OT_TAKE(lq_items, unsigned long long, max_layer_jobs(c) + kQueueMargin)
     OT_TAKE(g, int32_t, B * (n + 1))
     OT_TAKE(vdone, int32_t, B)
     OT_TAKE(status, int32_t, 1)
@@ -117,7 +111,7 @@ struct Params {            // by-value kernel parameters
     int V, H, n, k, kk, Dcap, max_depth, B;
     float delta;
     int aligned;
-    int q_capacity, lq_capacity;
+    int q_capacity;
 };
 
 __device__ __forceinline__ SeqWork seq_work(const Workspace& w, const Params& p, int b) {
@@ -146,12 +140,17 @@ __device__ __forceinline__ TreeOut tree_out(const opt_tree_out& o, const Params&
 }
 
 // Queue item: bit 63 valid | b (15 bits) | layer d (9) | rows in the layer (9) | frontier slot (8) |
-// table row of the node to expand (22).  Packing the row index spares the consumer of an item a
-// dependent load of the node's token.
+// table row of the node to expand (22).  A second word at the same queue position carries the
+// node's path value (bit 63 valid; a path value is never negative).  Both words validate themselves,
+// so a row can be expanded from them alone and the publisher needs no fence before writing them.
 constexpr int kMaxTableRows = 1 << 22;
 __device__ __forceinline__ unsigned long long item_encode(int b, int d, int fsize, int slot, int row) {
     return (1ull << 63) | ((unsigned long long)b << 48) | ((unsigned long long)d << 39) |
            ((unsigned long long)fsize << 30) | ((unsigned long long)slot << 22) | (unsigned long long)row;
+}
+
+__device__ __forceinline__ unsigned long long phat_word(double p) {
+    return (1ull << 63) | (unsigned long long)__double_as_longlong(p);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -168,121 +167,132 @@ __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restri
             item = item_encode(i, 1, 1, 0, row_of(token, 0, p.H));
         }
         w.q_items[i] = item;
+        w.q_phat[i] = i < p.B ? phat_word(1.0) : 0ull;        // the root counts as factor 1
     }
-    if (i < p.lq_capacity) w.lq_items[i] = 0ull;
     if (i < p.B) {
         int32_t* st = w.st + (size_t)i * 8;
-        st[kStDone] = 0; st[kStNR] = 0; st[kStUpdated] = 0;
+        st[kStDone] = 0; st[kStNR] = 0;
         w.E_prev[i] = 0.0;
     }
-    if (i == 0) {
-        w.q_ctl[kQHead] = 0; w.q_ctl[kQTail] = p.B; w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0;
-        w.q_ctl[kLQHead] = 0; w.q_ctl[kLQTail] = 0;
-    }
+    if (i == 0) { w.q_ctl[kQHead] = 0; w.q_ctl[kQTail] = p.B; w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; }
 }
 
 // Source of the tree build: rows come from the global work queue.
 struct BuildSource {
     Workspace w; Params p;
     const uint16_t* draft;
-    __device__ bool next(RowDesc& d) {
+    __device__ long long claim(int) {
         const int idx = atomicAdd(&w.q_ctl[kQHead], 1);
-        if (idx >= p.q_capacity) return false;
-        unsigned long long item = ld_acquire_u64(&w.q_items[idx]);
-        if (!(item >> 63)) {
-            const long long t0 = clock64();
-            for (;;) {
-                if (ld_acquire_s32(&w.q_ctl[kQDone])) return false;
-                item = ld_acquire_u64(&w.q_items[idx]);
-                if (item >> 63) break;
-                if (clock64() - t0 > kWaitCycles) { set_status(w.status, kErrTimeout); return false; }
-                __nanosleep(64);
-            }
-        }
+        return idx < p.q_capacity ? idx : -1;
+    }
+    // Both words of the item validate themselves; the shared "all done" flag is looked at only when
+    // check_done is set, so that a thousand waiting lanes do not pile onto one L2 line.
+    __device__ int poll(long long idx, RowDesc& d, bool check_done) {
+        const unsigned long long item = ld_relaxed_u64(&w.q_items[idx]), ph = ld_relaxed_u64(&w.q_phat[idx]);
+        if (!((item & ph) >> 63)) return check_done && ld_acquire_s32(&w.q_ctl[kQDone]) ? -1 : 0;
         d.b = (int)((item >> 48) & 0x7FFFu); d.d = (int)((item >> 39) & 0x1FFu);
         d.fsize = (int)((item >> 30) & 0x1FFu); d.slot = (int)((item >> 22) & 0xFFu);
+        d.pphat = __longlong_as_double((long long)(ph & 0x7FFFFFFFFFFFFFFFull));
         int row = (int)(item & 0x3FFFFFu);
         if (row >= p.H) { set_status(w.status, kErrInternal); row = 0; }
         d.row = draft + (size_t)row * p.V;
-        return true;
+        return 1;
     }
 };
 
-// Layer job: bit 63 valid | b (15 bits) | layer d (9) | rows in the layer (9).
-__device__ __forceinline__ unsigned long long job_encode(int b, int d, int fsize) {
-    return (1ull << 63) | ((unsigned long long)b << 48) | ((unsigned long long)d << 39) | ((unsigned long long)fsize << 30);
-}
-
-// Sink of the tree build.  Finisher warps: candidates' path values (Eq. 2); the row that completes
-// its layer posts a layer job.  Layer warp: takes jobs, does the layer selection / loop test, and
-// either publishes the next layer's rows or leaves the packed tree.
+// Sink of the tree build.  Finisher warps: candidates' path values (Eq. 2) and the layer's row
+// counter.  Layer warp: the layer warp of CTA c owns sequences c, c + gridDim.x, ...; it watches
+// their row counters, and when a layer is complete does the layer selection, publishes the next
+// layer's rows, brings the running top-n up to date and applies the loop test of Algorithm 1.
 struct BuildSink {
     Workspace w; Params p; opt_tree_out out;
     __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch&) {
         const int lane = threadIdx.x & 31;
         const SeqWork sw = seq_work(w, p, d.b);
-        const double parent_phat = d.d == 1 ? 1.0 : __ldcg(&sw.T_phat[(size_t)(d.d - 2) * p.n + d.slot]);   // root: factor 1
         if (lane < p.k) {
-            sw.cand_phat[d.slot * p.k + lane] = lane < r.kk ? parent_phat * r.p : -1.0;
+            sw.cand_phat[d.slot * p.k + lane] = lane < r.kk ? d.pphat * r.p : -1.0;
             sw.cand_tok[d.slot * p.k + lane] = r.tok;
         }
-        __threadfence();
         __syncwarp();
-        if (lane == 0 && atomicAdd(&sw.st[kStDone], 1) == d.fsize - 1) {
-            __threadfence();
-            const int pos = atomicAdd(&w.q_ctl[kLQTail], 1);
-            if (pos < p.lq_capacity) st_release_u64(&w.lq_items[pos], job_encode(d.b, d.d, d.fsize));
-            else set_status(w.status, kErrInternal);
-        }
+        if (lane == 0) atom_add_release_s32(&sw.st[kStDone], 1);     // orders the warp's candidates before the count;
+                                                                     // the count runs on over the layers of a build
     }
-    // Queue items for the rows of layer d+1 (the nodes select_layer_warp just chose).
-    __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl) {
+    // Queue items for the rows of layer d+1 (the nodes select_layer_warp just chose), at queue
+    // positions pos .. pos+nl reserved beforehand.
+    __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl, int pos) {
         const int lane = threadIdx.x & 31;
-        int pos = 0;
-        if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
-        pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
-        __threadfence();                                   // the layer's nodes before its queue items
         for (int i = lane; i < nl; i += 32) {
             int token = ls.ltok[i];
             if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
-            if (pos + i < p.q_capacity) st_relaxed_u64(&w.q_items[pos + i], item_encode(b, d + 1, nl, i, row_of(token, d, p.H)));
-            else set_status(w.status, kErrInternal);
+            if (pos + i < p.q_capacity) {
+                st_relaxed_u64(&w.q_phat[pos + i], (1ull << 63) | (ls.lkeys[i] - 1ull));
+                st_relaxed_u64(&w.q_items[pos + i], item_encode(b, d + 1, nl, i, row_of(token, d, p.H)));
+            } else {
+                set_status(w.status, kErrInternal);
+            }
         }
         __syncwarp();
     }
     __device__ void layer_loop(LayerScratch& ls) {
         const int lane = threadIdx.x & 31;
-        for (;;) {
-            unsigned long long job = 0ull;
-            if (lane == 0) {
-                const int idx = atomicAdd(&w.q_ctl[kLQHead], 1);
-                if (idx < p.lq_capacity) {
-                    const long long t0 = clock64();
-                    for (;;) {
-                        job = ld_acquire_u64(&w.lq_items[idx]);
-                        if (job >> 63) break;
-                        if (ld_acquire_s32(&w.q_ctl[kQDone])) { job = 0ull; break; }
-                        if (clock64() - t0 > kWaitCycles) { set_status(w.status, kErrTimeout); job = 0ull; break; }
-                        __nanosleep(200);
+        constexpr int kOwn = 4;                            // sequences one layer warp follows at a time
+        for (int b0 = blockIdx.x; b0 < p.B; b0 += kOwn * gridDim.x) {
+            // layer in flight (0 = finished / none), its row count, rows expected in all layers so far
+            int cur_d[kOwn], cur_f[kOwn], cur_tot[kOwn];
+            int live = 0;
+#pragma unroll
+            for (int q = 0; q < kOwn; ++q) {
+                const bool has = b0 + q * (int)gridDim.x < p.B;
+                cur_d[q] = has ? 1 : 0; cur_f[q] = 1; cur_tot[q] = 1; live += has ? 1 : 0;
+            }
+            long long t0 = clock64();
+            while (live > 0) {
+                bool progressed = false;
+#pragma unroll
+                for (int q = 0; q < kOwn; ++q) {
+                    if (cur_d[q] == 0) continue;
+                    const int b = b0 + q * (int)gridDim.x;
+                    const SeqWork sw = seq_work(w, p, b);
+                    int done = 0;
+                    if (lane == 0) done = ld_acquire_s32(&sw.st[kStDone]);
+                    done = __shfl_sync(0xFFFFFFFFu, done, 0);
+                    if (done < cur_tot[q]) continue;
+                    progressed = true;
+                    const int d = cur_d[q], fsize = cur_f[q];
+                    const int nvalid = fsize * p.kk, nl = nvalid < p.n ? nvalid : p.n;
+                    // Without a threshold the loop test only looks at the depth: the next layer's rows
+                    // can go out before the running top-n is brought up to date.
+                    const bool early = d < p.Dcap && p.delta == -INFINITY;
+                    int pos = 0;
+                    if (early) {                           // reserve the queue positions while the candidates load
+                        if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
                     }
+                    select_layer_warp(ls, sw, d, fsize, p.n, p.k, p.kk);
+                    if (early) {
+                        pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
+                        publish_layer(ls, b, d, nl, pos);
+                    }
+                    const bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta,
+                                                          w.status);
+                    if (more && !early) {
+                        if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
+                        pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
+                        publish_layer(ls, b, d, nl, pos);
+                    }
+                    if (more) { cur_d[q] = d + 1; cur_f[q] = nl; cur_tot[q] += nl; }
+                    else {
+                        cur_d[q] = 0; --live;
+                        __threadfence();
+                        if (lane == 0 && atomicAdd(&w.q_ctl[kQFinished], 1) == p.B - 1) st_release_s32(&w.q_ctl[kQDone], 1);
+                    }
+                    __syncwarp();
+                }
+                if (progressed) t0 = clock64();
+                else {
+                    if (clock64() - t0 > kWaitCycles) { set_status(w.status, kErrTimeout); return; }
+                    __nanosleep(100);
                 }
             }
-            job = __shfl_sync(0xFFFFFFFFu, job, 0);
-            if (!(job >> 63)) return;
-            const int b = (int)((job >> 48) & 0x7FFFu), d = (int)((job >> 39) & 0x1FFu), fsize = (int)((job >> 30) & 0x1FFu);
-            const SeqWork sw = seq_work(w, p, b);
-            const int nl = select_layer_warp(ls, sw, d, fsize, p.n, p.k, p.kk);
-            // Without a threshold the loop test only looks at the depth: the next layer's rows can
-            // go out before the running top-n is brought up to date.
-            const bool early = d < p.Dcap && p.delta == -INFINITY;
-            if (early) publish_layer(ls, b, d, nl);
-            const bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta, w.status);
-            if (more && !early) publish_layer(ls, b, d, nl);
-            if (!more && !early) {
-                __threadfence();
-                if (lane == 0 && atomicAdd(&w.q_ctl[kQFinished], 1) == p.B - 1) st_release_s32(&w.q_ctl[kQDone], 1);
-            }
-            __syncwarp();
         }
     }
 };
@@ -300,14 +310,16 @@ build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, opt_tree
 
 // The row step alone over a list of rows (static round-robin over the CTAs).
 struct ListSource {
-    const uint16_t* logits; const int32_t* rows; int nrows, V, H, next_idx, stride; int* status;
-    __device__ bool next(RowDesc& d) {
-        if (next_idx >= nrows) return false;
-        int r = rows[next_idx];
-        if (r < 0 || r >= H) { set_status(status, kErrInternal); r = 0; }
-        d.row = logits + (size_t)r * V; d.slot = next_idx; d.b = d.d = 0; d.fsize = 1;
-        next_idx += stride;
-        return true;
+    const uint16_t* logits; const int32_t* rows; int nrows, V, H, first, stride; int* status;
+    __device__ long long claim(int r) {
+        const long long idx = (long long)first + (long long)r * stride;
+        return idx < nrows ? idx : -1;
+    }
+    __device__ int poll(long long idx, RowDesc& d, bool) {
+        int row = rows[idx];
+        if (row < 0 || row >= H) { set_status(status, kErrInternal); row = 0; }
+        d.row = logits + (size_t)row * V; d.slot = (int)idx; d.b = d.d = 0; d.fsize = 1;
+        return 1;
     }
 };
 struct ListSink {
@@ -484,7 +496,7 @@ struct opt_tree_ctx {
     size_t bytes;
     int device;
     int grid;              // resident CTAs of the persistent kernels (SMs x occupancy)
-    int q_capacity, lq_capacity;
+    int q_capacity;
     int64_t launches;
 };
 
@@ -507,7 +519,6 @@ ot::Params make_params(const opt_tree_ctx* ctx, const void* table, float delta) 
     p.max_depth = c.max_depth;
     p.B = 0;
     p.q_capacity = ctx->q_capacity;
-    p.lq_capacity = ctx->lq_capacity;
     p.delta = delta;
     p.aligned = ((reinterpret_cast<uintptr_t>(table) & 15u) == 0 && (c.V % 8) == 0) ? 1 : 0;
     return p;
@@ -544,7 +555,6 @@ int opt_tree_create(opt_tree_ctx** out, const opt_tree_config* cfg) {
     }
     ot::carve(*cfg, static_cast<char*>(ctx->base), &ctx->ws);
     ctx->q_capacity = (int)(ot::max_items(*cfg) + ot::kQueueMargin);
-    ctx->lq_capacity = (int)(ot::max_layer_jobs(*cfg) + ot::kQueueMargin);
     bool ok = cudaMemset(ctx->base, 0, ctx->bytes) == cudaSuccess;
     ok = ok && cudaFuncSetAttribute(ot::build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)sizeof(ot::CtaSmem)) == cudaSuccess;
@@ -579,7 +589,7 @@ int opt_tree_build(opt_tree_ctx* ctx, const void* draft, const int32_t* root_tok
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     ot::Params p = make_params(ctx, draft, delta);
     p.B = B;
-    ot::init_build_kernel<<<((ctx->q_capacity > ctx->lq_capacity ? ctx->q_capacity : ctx->lq_capacity) + 255) / 256, 256, 0, st>>>(ctx->ws, p, root_token);
+    ot::init_build_kernel<<<(ctx->q_capacity + 255) / 256, 256, 0, st>>>(ctx->ws, p, root_token);
     ot::build_kernel<<<ctx->grid, ot::kThreads, sizeof(ot::CtaSmem), st>>>(
         ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
     ctx->launches += 2;

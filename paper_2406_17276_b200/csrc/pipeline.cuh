@@ -1,17 +1,18 @@
 // The persistent, warp-specialised row pipeline of one CTA.
 //
-//   fetcher warp    asks a Source for row descriptors, up to kDesc rows ahead of the consumers, so
-//                   that the latency of obtaining work (a queue pop, an index load) is hidden;
+//   fetcher warp    asks a Source for row descriptors, several at a time and ahead of the
+//                   consumers, so that the latency of obtaining work (a queue pop, an index load)
+//                   is hidden, and hands them on in the order in which they become known;
 //   issuer warp     streams each described row's chunks into the ring (bulk async copies) as
 //                   stages are handed back;
 //   consumer warps  make the fused pass over each row (row_topk.cuh), then hand the row's
 //                   per-thread maxima and partial sums to a finisher through a slot and go
 //                   straight on to the next row;
 //   finisher warps  row r goes to finisher r mod kFinishers: it computes the row's winners and
-//                   gives them to a Sink (for the tree build: candidates' path values, and a
-//                   layer job once a layer's last row is in);
-//   layer warp      runs Sink::layer_loop (for the tree build: takes layer jobs from a queue,
-//                   selects the next layer and publishes its rows).
+//                   gives them to a Sink (for the tree build: candidates' path values and the
+//                   layer's row counter);
+//   layer warp      runs Sink::layer_loop (for the tree build: watches the row counters of its
+//                   sequences, selects each next layer and publishes its rows).
 //
 // The chunks of consecutive rows form one stream: chunk g lives in stage g % kStages and is the
 // (g / kStages)-th use of that stage, which fixes every mbarrier parity; likewise row r uses
@@ -36,24 +37,61 @@ __device__ __forceinline__ void pipeline_init(CtaSmem& s) {
 }
 
 // ---- fetcher warp ------------------------------------------------------------------------------
-// Source::next(RowDesc&) is called by lane 0 only and returns false when there is no more work.
+// Obtaining a row costs global-memory round trips (a queue pop and its item, an index load) that
+// take about as long as streaming the row, so kFetchLanes lanes hold one ticket each and poll
+// concurrently; the warp stays converged in one polling loop so that the lanes' round trips
+// overlap.  Rows are handed on in the order in which they become known (the a-th known row goes to
+// descriptor a % kDesc), never in ticket order: a ticket whose item is published late must not hold
+// up a row that is ready.  Tickets are only taken while fewer than kDesc rows are between "ticket
+// taken" and "descriptor read by the consumers", which bounds what a CTA keeps from the others.
+//   Source::claim(i)          ticket for this CTA's i-th claim, or a negative value: no more work
+//   Source::poll(ticket, dsc) 1: descriptor filled, 0: not yet, -1: no more work
+// Once a Source has said "no more work" no ticket of this CTA can still turn into a row.
+constexpr int kFetchLanes = 4;
 template <class Source>
 __device__ void fetcher_role(CtaSmem& s, Source& src, int* status) {
     const int lane = threadIdx.x & 31;
-    for (int r = 0;; ++r) {
-        const int e = r % kDesc;
-        if (r >= kDesc && !mbar_wait_warp(&s.desc_empty[e], (uint32_t)((r / kDesc) - 1) & 1u, status)) return;
-        int go = 0;
-        if (lane == 0) {
-            RowDesc dsc;
-            dsc.row = nullptr; dsc.b = dsc.d = dsc.slot = dsc.fsize = 0;
-            go = src.next(dsc) ? 1 : 0;
-            dsc.stop = go ? 0 : 1;
-            s.desc[e] = dsc;
-            mbar_arrive(&s.desc_full[e]);                      // release: publishes the descriptor
+    const unsigned below = (1u << lane) - 1u;
+    bool holding = false;                 // this lane has a ticket
+    long long ticket = 0;
+    int claimed = 0, known = 0, consumed = 0;      // warp-uniform counts of this CTA's rows
+    long long t0 = clock64();
+    for (int turn = 0;; ++turn) {
+        // rows whose descriptors the consumers have let go of
+        while (consumed < known && mbar_test_wait(&s.desc_empty[consumed % kDesc], (uint32_t)(consumed / kDesc) & 1u)) ++consumed;
+        // new tickets, as far as the bound allows
+        const bool want = lane < kFetchLanes && !holding;
+        const unsigned wm = __ballot_sync(0xFFFFFFFFu, want);
+        const int my_claim = claimed + __popc(wm & below);
+        const bool take = want && my_claim - consumed < kDesc;
+        if (take) { ticket = src.claim(my_claim); holding = true; }
+        claimed += __popc(__ballot_sync(0xFFFFFFFFu, take));
+        // one poll per held ticket
+        RowDesc dsc;
+        dsc.row = nullptr; dsc.pphat = 0.0; dsc.b = dsc.d = dsc.slot = dsc.fsize = 0; dsc.stop = 0;
+        int got = 0;
+        if (holding) got = ticket < 0 ? -1 : src.poll(ticket, dsc, (turn & 15) == 15);
+        const unsigned rm = __ballot_sync(0xFFFFFFFFu, got > 0), em = __ballot_sync(0xFFFFFFFFu, got < 0);
+        if (got > 0) {
+            const int a = known + __popc(rm & below);
+            s.desc[a % kDesc] = dsc;
+            mbar_arrive(&s.desc_full[a % kDesc]);              // release: publishes the descriptor
+            holding = false;
         }
-        go = __shfl_sync(0xFFFFFFFFu, go, 0);
-        if (!go) return;
+        known += __popc(rm);
+        if (em) {                                              // no more work: one stop marker after the last row
+            if (lane == __ffs(em) - 1) {
+                dsc.stop = 1;
+                s.desc[known % kDesc] = dsc;
+                mbar_arrive(&s.desc_full[known % kDesc]);
+            }
+            return;
+        }
+        if (rm) t0 = clock64();
+        else {
+            if ((turn & 63) == 63 && clock64() - t0 > kWaitCycles) { set_status(status, kErrTimeout); return; }
+            __nanosleep(100);
+        }
     }
 }
 

@@ -33,7 +33,7 @@ constexpr int kStages = 4;                         // ring depth (128 KB)
 constexpr int kSlots = kFinishers + 2;             // finished rows waiting for / held by finishers
 constexpr int kCandCap = 128;                      // candidate list capacity per row
 constexpr int kMaxFlag = 64;                       // flagged threads the fast finisher accepts
-constexpr int kDesc = 4;                           // row descriptors fetched ahead
+constexpr int kDesc = 4;                           // rows a CTA may hold between ticket and descriptor read
 constexpr int kPerLane = kConsumers / 32;          // per-thread results one finisher lane handles (16)
 
 constexpr float kLog2e = 1.44269504088896340736f;
@@ -45,14 +45,16 @@ constexpr int kExpLimit = 15000;                   // |E| beyond this: magnitude
 // Fetcher -> issuer / consumers: which row the next chunks of the stream belong to.
 struct RowDesc {
     const uint16_t* row;      // global address of the row's first logit
+    double pphat;             // tree build: path value of the node being expanded
     int b, d, slot;           // caller's coordinates (sequence, layer, frontier slot / list index)
     int fsize;                // rows in this (sequence, layer)
     int stop;                 // 1: no more rows, shut the pipeline down
 };
 
 // Consumers -> finisher: what the fused pass leaves behind for one row.  Thread t's sum is
-// relative to the exponent of its warp, warpE[t / 32].
-struct RowSlot {
+// relative to the exponent of its warp, warpE[t / 32].  The finisher reads tsum and tkey with
+// 16-byte loads, so every slot of the array must start on a 16-byte boundary.
+struct alignas(16) RowSlot {
     float tsum[kConsumers];
     uint16_t tkey[kConsumers];     // per-thread maximum as an ordered key
     int warpE[kConsumerWarps];
@@ -76,6 +78,8 @@ struct LayerScratch {              // private to the layer warp of a CTA
     int ltok[kMaxN];                           // tokens of the new layer, slot order
     int hist[256];
 };
+
+static_assert(sizeof(RowSlot) % 16 == 0, "slots must keep 16-byte alignment in an array");
 
 struct alignas(128) CtaSmem {
     uint16_t stage[kStages][kChunkElems];

@@ -115,9 +115,9 @@ struct SeqWork {
     double* T_phat;        // [D*n]
     int32_t* R;            // [2][n]   running top-n as gids in ascending order, double-buffered by layer parity
     double* E_prev;        // [1]      E of Algorithm 1
-    int32_t* st;           // [8]      1: rows finished in this layer, 2: |R|, 3: last layer folded into R
+    int32_t* st;           // [8]      1: rows finished since the build began, 2: |R|
 };
-enum { kStDone = 1, kStNR = 2, kStUpdated = 3 };
+enum { kStDone = 1, kStNR = 2 };
 
 struct TreeOut {           // mirrors opt_tree_out, pointers offset to the sequence
     int32_t *token, *parent, *depth;
@@ -129,8 +129,7 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
 
 // Layer job, first half.  After all rows of layer d (1-based) of one sequence are expanded: the
 // next layer = the nl candidates of largest path value, stored in candidate-index order (nodes
-// gid0 .. gid0+nl of T; tokens and keys also left in s.ltok / s.lkeys).  Resets the sequence's
-// row counter.  Whole layer warp; s is its scratch; fsize = rows of the layer.  Returns nl.
+// gid0 .. gid0+nl of T; tokens and keys also left in s.ltok / s.lkeys).  Whole layer warp; s is its scratch; fsize = rows of the layer.  Returns nl.
 __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int fsize, int n, int k, int kk) {
     const int lane = threadIdx.x & 31;
     int* hist = s.hist;
@@ -176,16 +175,14 @@ __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int f
             s.lkeys[pos] = key;
         });
     }
-    if (lane == 0) w.st[kStDone] = 0;
     __syncwarp();
     return nl;
 }
 
 // Layer job, second half: the running top-n and E_sub(T, n) with the new layer (left in s by
 // select_layer_warp), the loop test of Algorithm 1, and the packed tree if the sequence is
-// finished.  Layer d's update must follow layer d-1's (they may run on different CTAs): the
-// sequence's st[kStUpdated] holds the last layer whose update is complete.  Returns true if the
-// sequence continues with layer d+1, false if it is finished (outputs written) or a wait expired.
+// finished.  All layers of a sequence are handled by the same warp, in order.  Returns true if the
+// sequence continues with layer d+1, false if it is finished (outputs written).
 __device__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
                                     int max_depth, float delta, int* status) {
     const int lane = threadIdx.x & 31;
@@ -193,17 +190,6 @@ __device__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const Tre
     const int gid0 = (d - 1) * n;
     unsigned long long thr;
     int need_eq;
-    if (d > 1) {
-        int ok = 1;
-        if (lane == 0) {
-            const long long t0 = clock64();
-            while (ld_acquire_s32(&w.st[kStUpdated]) < d - 1) {
-                if (clock64() - t0 > kWaitCycles) { set_status(status, kErrTimeout); ok = 0; break; }
-                __nanosleep(100);
-            }
-        }
-        if (!__shfl_sync(0xFFFFFFFFu, ok, 0)) return false;
-    }
     const int nR_old = d == 1 ? 0 : __ldcg(&w.st[kStNR]);
     const double eprev = d == 1 ? 0.0 : __ldcg(w.E_prev);
 
@@ -241,9 +227,7 @@ __device__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const Tre
         w.st[kStNR] = nR;
         *w.E_prev = esub;
     }
-    __threadfence();
     __syncwarp();
-    if (lane == 0) st_release_s32(&w.st[kStUpdated], d);
     if (more) return true;
 
     // --- pack: T_opt = the running top-n, already in (depth, parent's index, sibling rank) order ---
