@@ -25,18 +25,19 @@ __device__ __forceinline__ int row_of(int token, int depth, int H) {
 // ------------------------------------------------------------------------------------------------
 struct Workspace {
     // build
-    double* cand_phat;     // [B][n*k]
-    int32_t* cand_tok;     // [B][n*k]
+    double* cand_phat;     // [B][cand_stride]
+    int32_t* cand_tok;     // [B][cand_stride]
     int32_t* T_tok;        // [B][D*n]
     int32_t* T_par;        // [B][D*n]
     double* T_phat;        // [B][D*n]
     int32_t* R;            // [B][2][n]
     double* E_prev;        // [B]
     int32_t* st;           // [B][8]
-    // work queue of the build: one item per (sequence, layer, frontier slot)
-    unsigned long long* q_items;   // [q_capacity]
-    unsigned long long* q_phat;    // [q_capacity]  bit 63 valid | bits of the parent's path value (a double >= 0)
-    int32_t* q_ctl;        // [8]  0: head (next to claim), 1: tail (published), 2: sequences finished, 3: all done
+    // row mailboxes of the build: one per CTA, filled by the layer warps, never wrapped within a build
+    unsigned long long* mb_items;  // [grid][mcap]  one item per (sequence, layer, frontier slot)
+    unsigned long long* mb_phat;   // [grid][mcap]  bit 63 valid | bits of the node's path value (a double >= 0)
+    int32_t* mb_tail;      // [grid]  entries reserved so far
+    int32_t* q_ctl;        // [8]  2: sequences finished, 3: all done
     // verify
     int32_t* g;            // [B][n+1]  target argmax after the root (0) and after node i (i+1)
     int32_t* vdone;        // [B]
@@ -48,17 +49,20 @@ struct Workspace {
     uint64_t* o_mask; int32_t* o_pos;
     int32_t *o_alen, *o_atok, *o_anode, *o_next;
 };
-enum { kQHead = 0, kQTail = 1, kQFinished = 2, kQDone = 3 };
+enum { kQFinished = 2, kQDone = 3 };
 
-constexpr int kQueueMargin = 4096;          // room for one over-claim per resident CTA
+constexpr int kMaxGrid = 4096;              // CTAs of the persistent kernels (SMs x occupancy) this layout supports
 
-static size_t max_items(const opt_tree_config& c) {
-    const size_t n = c.n, kk = c.k < c.V ? c.k : c.V, Dcap = c.max_depth < c.n ? c.max_depth : c.n;
-    size_t per_seq = 1;
-    if (Dcap >= 2) per_seq += kk < n ? kk : n;
-    if (Dcap >= 3) per_seq += (Dcap - 2) * n;
-    return per_seq * (size_t)c.max_batch;
+// Rows of one layer go to consecutive CTAs, so a CTA receives at most ceil(n / grid) rows per
+// (sequence, layer); its mailbox holds every row it can be sent during one build.
+static size_t mailbox_capacity(const opt_tree_config& c, int grid) {
+    const size_t Dcap = c.max_depth < c.n ? c.max_depth : c.n;
+    // + 8: a fetcher takes a few tickets beyond the last row it will ever get; those must stay inside
+    return (size_t)c.max_batch * Dcap * (((size_t)c.n + grid - 1) / grid) + 8;
 }
+
+// Entries per sequence in the candidate arrays: n*k rounded up to a multiple of four (16-byte vectors).
+static size_t cand_stride(int n, int k) { return ((size_t)n * k + 3) & ~(size_t)3; }
 
 struct Layout {
     size_t total = 0;
@@ -69,21 +73,23 @@ struct Layout {
     }
 };
 
-static size_t carve(const opt_tree_config& c, char* base, Workspace* w) {
-    const size_t B = c.max_batch, n = c.n, k = c.k, D = c.max_depth, W = (c.n + 63) / 64;
+static size_t carve(const opt_tree_config& c, int grid, char* base, Workspace* w) {
+    const size_t B = c.max_batch, n = c.n, D = c.max_depth, W = (c.n + 63) / 64;
+    const size_t cs = cand_stride(c.n, c.k);
     Layout L;
     size_t o;
 #define OT_TAKE(field, T, count) o = L.take<T>(count); if (w) w->field = reinterpret_cast<T*>(base + o);
-    OT_TAKE(cand_phat, double, B * n * k)
-    OT_TAKE(cand_tok, int32_t, B * n * k)
+    OT_TAKE(cand_phat, double, B * cs)
+    OT_TAKE(cand_tok, int32_t, B * cs)
     OT_TAKE(T_tok, int32_t, B * D * n)
     OT_TAKE(T_par, int32_t, B * D * n)
     OT_TAKE(T_phat, double, B * D * n)
     OT_TAKE(R, int32_t, B * 2 * n)
     OT_TAKE(E_prev, double, B)
     OT_TAKE(st, int32_t, B * 8)
-    OT_TAKE(q_items, unsigned long long, max_items(c) + kQueueMargin)
-    OT_TAKE(q_phat, unsigned long long, max_items(c) + kQueueMargin)
+    OT_TAKE(mb_items, unsigned long long, mailbox_capacity(c, grid) * grid)
+    OT_TAKE(mb_phat, unsigned long long, mailbox_capacity(c, grid) * grid)
+    OT_TAKE(mb_tail, int32_t, grid)
     OT_TAKE(q_ctl, int32_t, 8)
     OT_TAKE(g, int32_t, B * (n + 1))
     OT_TAKE(vdone, int32_t, B)
@@ -111,13 +117,13 @@ struct Params {            // by-value kernel parameters
     int V, H, n, k, kk, Dcap, max_depth, B;
     float delta;
     int aligned;
-    int q_capacity;
+    int mcap, grid, cstride;
 };
 
 __device__ __forceinline__ SeqWork seq_work(const Workspace& w, const Params& p, int b) {
     SeqWork s;
-    s.cand_phat = w.cand_phat + (size_t)b * p.n * p.k;
-    s.cand_tok = w.cand_tok + (size_t)b * p.n * p.k;
+    s.cand_phat = w.cand_phat + (size_t)b * p.cstride;
+    s.cand_tok = w.cand_tok + (size_t)b * p.cstride;
     s.T_tok = w.T_tok + (size_t)b * p.max_depth * p.n;
     s.T_par = w.T_par + (size_t)b * p.max_depth * p.n;
     s.T_phat = w.T_phat + (size_t)b * p.max_depth * p.n;
@@ -139,14 +145,14 @@ __device__ __forceinline__ TreeOut tree_out(const opt_tree_out& o, const Params&
     return t;
 }
 
-// Queue item: bit 63 valid | b (15 bits) | layer d (9) | rows in the layer (9) | frontier slot (8) |
-// table row of the node to expand (22).  A second word at the same queue position carries the
-// node's path value (bit 63 valid; a path value is never negative).  Both words validate themselves,
-// so a row can be expanded from them alone and the publisher needs no fence before writing them.
+// Mailbox item: bit 63 valid | b (15 bits) | layer d (9) | frontier slot (8) | table row of the node to
+// expand (22).  A second word at the same mailbox position carries the node's path value (bit 63
+// valid; a path value is never negative).  Both words validate themselves, so a row can be expanded
+// from them alone and the publisher needs no fence before writing them.
 constexpr int kMaxTableRows = 1 << 22;
-__device__ __forceinline__ unsigned long long item_encode(int b, int d, int fsize, int slot, int row) {
+__device__ __forceinline__ unsigned long long item_encode(int b, int d, int slot, int row) {
     return (1ull << 63) | ((unsigned long long)b << 48) | ((unsigned long long)d << 39) |
-           ((unsigned long long)fsize << 30) | ((unsigned long long)slot << 22) | (unsigned long long)row;
+           ((unsigned long long)slot << 22) | (unsigned long long)row;
 }
 
 __device__ __forceinline__ unsigned long long phat_word(double p) {
@@ -156,42 +162,47 @@ __device__ __forceinline__ unsigned long long phat_word(double p) {
 // ------------------------------------------------------------------------------------------------
 // Kernels
 // ------------------------------------------------------------------------------------------------
-// Clears the queue, publishes one root row per sequence and resets the per-sequence state.
+// Clears the mailboxes, sends the root row of sequence b to CTA b % grid and resets the per-sequence state.
 __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restrict__ root_token) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < p.q_capacity) {
-        unsigned long long item = 0ull;
-        if (i < p.B) {
-            int token = root_token[i];
+    if (i < p.grid * p.mcap) {
+        const int c = i / p.mcap, j = i - c * p.mcap;
+        const long long b = (long long)c + (long long)j * p.grid;         // the j-th root sent to CTA c
+        unsigned long long item = 0ull, ph = 0ull;
+        if (b < p.B) {
+            int token = root_token[b];
             if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
-            item = item_encode(i, 1, 1, 0, row_of(token, 0, p.H));
+            item = item_encode((int)b, 1, 0, row_of(token, 0, p.H));
+            ph = phat_word(1.0);                                          // the root counts as factor 1
         }
-        w.q_items[i] = item;
-        w.q_phat[i] = i < p.B ? phat_word(1.0) : 0ull;        // the root counts as factor 1
+        w.mb_items[i] = item;
+        w.mb_phat[i] = ph;
+    }
+    if (i < p.grid) w.mb_tail[i] = i < p.B ? (p.B - i + p.grid - 1) / p.grid : 0;
+    for (long long j = i; j < (long long)p.B * p.cstride; j += (long long)gridDim.x * blockDim.x) {
+        reinterpret_cast<unsigned long long*>(w.cand_phat)[j] = 0ull;
+        w.cand_tok[j] = 0;
     }
     if (i < p.B) {
         int32_t* st = w.st + (size_t)i * 8;
         st[kStDone] = 0; st[kStNR] = 0;
         w.E_prev[i] = 0.0;
     }
-    if (i == 0) { w.q_ctl[kQHead] = 0; w.q_ctl[kQTail] = p.B; w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; }
+    if (i == 0) { w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; }
 }
 
-// Source of the tree build: rows come from the global work queue.
+// Source of the tree build: the rows other CTAs' layer warps have put into this CTA's mailbox.
 struct BuildSource {
     Workspace w; Params p;
     const uint16_t* draft;
-    __device__ long long claim(int) {
-        const int idx = atomicAdd(&w.q_ctl[kQHead], 1);
-        return idx < p.q_capacity ? idx : -1;
-    }
-    // Both words of the item validate themselves; the shared "all done" flag is looked at only when
-    // check_done is set, so that a thousand waiting lanes do not pile onto one L2 line.
+    __device__ long long claim(int i) { return i < p.mcap ? (long long)blockIdx.x * p.mcap + i : -1; }
+    // Both words of an entry validate themselves; the "all done" flag is looked at only when
+    // check_done is set.
     __device__ int poll(long long idx, RowDesc& d, bool check_done) {
-        const unsigned long long item = ld_relaxed_u64(&w.q_items[idx]), ph = ld_relaxed_u64(&w.q_phat[idx]);
+        const unsigned long long item = ld_relaxed_u64(&w.mb_items[idx]), ph = ld_relaxed_u64(&w.mb_phat[idx]);
         if (!((item & ph) >> 63)) return check_done && ld_acquire_s32(&w.q_ctl[kQDone]) ? -1 : 0;
         d.b = (int)((item >> 48) & 0x7FFFu); d.d = (int)((item >> 39) & 0x1FFu);
-        d.fsize = (int)((item >> 30) & 0x1FFu); d.slot = (int)((item >> 22) & 0xFFu);
+        d.slot = (int)((item >> 22) & 0xFFu); d.fsize = 0;
         d.pphat = __longlong_as_double((long long)(ph & 0x7FFFFFFFFFFFFFFFull));
         int row = (int)(item & 0x3FFFFFu);
         if (row >= p.H) { set_status(w.status, kErrInternal); row = 0; }
@@ -209,24 +220,40 @@ struct BuildSink {
     __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch&) {
         const int lane = threadIdx.x & 31;
         const SeqWork sw = seq_work(w, p, d.b);
+        // Candidate words validate themselves (top bit; an absent child is all ones), so neither they nor
+        // the row count need a fence: the layer warp re-reads whatever it finds not yet written.
         if (lane < p.k) {
-            sw.cand_phat[d.slot * p.k + lane] = lane < r.kk ? d.pphat * r.p : -1.0;
-            sw.cand_tok[d.slot * p.k + lane] = r.tok;
+            unsigned long long* ph = reinterpret_cast<unsigned long long*>(sw.cand_phat) + d.slot * p.k + lane;
+            unsigned int* tk = reinterpret_cast<unsigned int*>(sw.cand_tok) + d.slot * p.k + lane;
+            *ph = lane < r.kk ? phat_word(d.pphat * r.p) : ~0ull;
+            *tk = lane < r.kk ? (0x80000000u | (unsigned int)r.tok) : ~0u;
         }
         __syncwarp();
-        if (lane == 0) atom_add_release_s32(&sw.st[kStDone], 1);     // orders the warp's candidates before the count;
-                                                                     // the count runs on over the layers of a build
+        if (lane == 0) atom_add_relaxed_s32(&sw.st[kStDone], 1);     // the count runs on over the layers of a build
     }
-    // Queue items for the rows of layer d+1 (the nodes select_layer_warp just chose), at queue
-    // positions pos .. pos+nl reserved beforehand.
-    __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl, int pos) {
+    // Rows of layer d+1 of sequence b go to consecutive CTAs starting at a CTA that depends on (b, d),
+    // so that one layer spreads over as many SMs as it has rows.  reserve_layer takes their mailbox
+    // positions (into ls.mpos), publish_layer writes the entries once the nodes are chosen.
+    __device__ int first_cta(int b, int d) const { return (int)(((unsigned)b * 37u + (unsigned)d * 61u) % (unsigned)p.grid); }
+    __device__ void reserve_layer(LayerScratch& ls, int b, int d, int nl) {
         const int lane = threadIdx.x & 31;
+        const int c0 = first_cta(b, d);
+        for (int i = lane; i < nl; i += 32) {
+            const int c = (c0 + i) % p.grid;
+            ls.mpos[i] = c * p.mcap + atomicAdd(&w.mb_tail[c], 1);
+        }
+        __syncwarp();
+    }
+    __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl) {
+        const int lane = threadIdx.x & 31;
+        const int c0 = first_cta(b, d);
         for (int i = lane; i < nl; i += 32) {
             int token = ls.ltok[i];
             if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
-            if (pos + i < p.q_capacity) {
-                st_relaxed_u64(&w.q_phat[pos + i], (1ull << 63) | (ls.lkeys[i] - 1ull));
-                st_relaxed_u64(&w.q_items[pos + i], item_encode(b, d + 1, nl, i, row_of(token, d, p.H)));
+            const int c = (c0 + i) % p.grid, pos = ls.mpos[i];
+            if (pos - c * p.mcap < p.mcap) {
+                st_relaxed_u64(&w.mb_phat[pos], (1ull << 63) | (ls.lkeys[i] - 1ull));
+                st_relaxed_u64(&w.mb_items[pos], item_encode(b, d + 1, i, row_of(token, d, p.H)));
             } else {
                 set_status(w.status, kErrInternal);
             }
@@ -263,21 +290,14 @@ struct BuildSink {
                     // Without a threshold the loop test only looks at the depth: the next layer's rows
                     // can go out before the running top-n is brought up to date.
                     const bool early = d < p.Dcap && p.delta == -INFINITY;
-                    int pos = 0;
-                    if (early) {                           // reserve the queue positions while the candidates load
-                        if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
-                    }
-                    select_layer_warp(ls, sw, d, fsize, p.n, p.k, p.kk);
-                    if (early) {
-                        pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
-                        publish_layer(ls, b, d, nl, pos);
-                    }
+                    if (early) reserve_layer(ls, b, d, nl);   // the mailbox positions, while the candidates load
+                    select_layer_warp(ls, sw, d, fsize, p.n, p.k, p.kk, w.status);
+                    if (early) publish_layer(ls, b, d, nl);
                     const bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta,
                                                           w.status);
                     if (more && !early) {
-                        if (lane == 0) pos = atomicAdd(&w.q_ctl[kQTail], nl);
-                        pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
-                        publish_layer(ls, b, d, nl, pos);
+                        reserve_layer(ls, b, d, nl);
+                        publish_layer(ls, b, d, nl);
                     }
                     if (more) { cur_d[q] = d + 1; cur_f[q] = nl; cur_tot[q] += nl; }
                     else {
@@ -496,7 +516,7 @@ struct opt_tree_ctx {
     size_t bytes;
     int device;
     int grid;              // resident CTAs of the persistent kernels (SMs x occupancy)
-    int q_capacity;
+    int mcap;
     int64_t launches;
 };
 
@@ -518,7 +538,9 @@ ot::Params make_params(const opt_tree_ctx* ctx, const void* table, float delta) 
     p.Dcap = c.max_depth < c.n ? c.max_depth : c.n;
     p.max_depth = c.max_depth;
     p.B = 0;
-    p.q_capacity = ctx->q_capacity;
+    p.mcap = ctx->mcap;
+    p.grid = ctx->grid;
+    p.cstride = (int)ot::cand_stride(c.n, c.k);
     p.delta = delta;
     p.aligned = ((reinterpret_cast<uintptr_t>(table) & 15u) == 0 && (c.V % 8) == 0) ? 1 : 0;
     return p;
@@ -532,9 +554,27 @@ int check_launch() { return cudaGetLastError() == cudaSuccess ? OPT_TREE_OK : OP
 
 extern "C" {
 
+// CTAs of the persistent kernels on the current device (one CTA of kThreads per SM as long as its
+// shared memory fits); 0 if there is no usable device.
+static int persistent_grid() {
+    int dev = 0, per_sm = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (cudaFuncSetAttribute(ot::build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::row_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ot::build_kernel, ot::kThreads, sizeof(ot::CtaSmem)) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    const int grid = per_sm * sms;
+    return grid >= 1 && grid <= ot::kMaxGrid ? grid : 0;
+}
+
 size_t opt_tree_workspace_bytes(const opt_tree_config* cfg) {
     if (!valid_cfg(cfg) || supported_cfg(cfg) != OPT_TREE_OK) return 0;
-    return ot::carve(*cfg, nullptr, nullptr);
+    int grid = persistent_grid();
+    if (grid == 0) grid = 148;                       // no device here: the size on a B200
+    return ot::carve(*cfg, grid, nullptr, nullptr);
 }
 
 int opt_tree_create(opt_tree_ctx** out, const opt_tree_config* cfg) {
@@ -547,25 +587,18 @@ int opt_tree_create(opt_tree_ctx** out, const opt_tree_config* cfg) {
     if (!ctx) return OPT_TREE_ERR_CUDA;
     ctx->cfg = *cfg;
     ctx->launches = 0;
-    ctx->bytes = ot::carve(*cfg, nullptr, nullptr);
+    ctx->grid = persistent_grid();
+    if (ctx->grid == 0) { delete ctx; return OPT_TREE_ERR_CUDA; }
+    ctx->mcap = (int)ot::mailbox_capacity(*cfg, ctx->grid);
+    ctx->bytes = ot::carve(*cfg, ctx->grid, nullptr, nullptr);
+    if ((long long)ctx->mcap * ctx->grid > 0x7FFFFFFFLL) { delete ctx; return OPT_TREE_ERR_UNSUPPORTED; }
     if (cudaGetDevice(&ctx->device) != cudaSuccess || cudaMalloc(&ctx->base, ctx->bytes) != cudaSuccess) {
         cudaGetLastError();
         delete ctx;
         return OPT_TREE_ERR_CUDA;
     }
-    ot::carve(*cfg, static_cast<char*>(ctx->base), &ctx->ws);
-    ctx->q_capacity = (int)(ot::max_items(*cfg) + ot::kQueueMargin);
-    bool ok = cudaMemset(ctx->base, 0, ctx->bytes) == cudaSuccess;
-    ok = ok && cudaFuncSetAttribute(ot::build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)sizeof(ot::CtaSmem)) == cudaSuccess;
-    ok = ok && cudaFuncSetAttribute(ot::row_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)sizeof(ot::CtaSmem)) == cudaSuccess;
-    int per_sm = 0, sms = 0;
-    ok = ok && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ot::build_kernel, ot::kThreads, sizeof(ot::CtaSmem)) == cudaSuccess;
-    ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device) == cudaSuccess;
-    ctx->grid = per_sm * sms;
-    ok = ok && ctx->grid >= 1 && ctx->grid <= ot::kQueueMargin;
-    if (!ok) {
+    ot::carve(*cfg, ctx->grid, static_cast<char*>(ctx->base), &ctx->ws);
+    if (cudaMemset(ctx->base, 0, ctx->bytes) != cudaSuccess) {
         cudaGetLastError();
         cudaFree(ctx->base);
         delete ctx;
@@ -589,7 +622,8 @@ int opt_tree_build(opt_tree_ctx* ctx, const void* draft, const int32_t* root_tok
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     ot::Params p = make_params(ctx, draft, delta);
     p.B = B;
-    ot::init_build_kernel<<<(ctx->q_capacity + 255) / 256, 256, 0, st>>>(ctx->ws, p, root_token);
+    const long long init_threads = (long long)ctx->grid * ctx->mcap > B ? (long long)ctx->grid * ctx->mcap : B;
+    ot::init_build_kernel<<<(unsigned)((init_threads + 255) / 256), 256, 0, st>>>(ctx->ws, p, root_token);
     ot::build_kernel<<<ctx->grid, ot::kThreads, sizeof(ot::CtaSmem), st>>>(
         ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
     ctx->launches += 2;

@@ -68,14 +68,15 @@ struct FinScratch {                // private to one finisher warp
     int cand_count;
 };
 
-struct LayerScratch {              // private to the layer warp of a CTA
-    unsigned long long keys[1024];             // staged candidate keys, then the keys of R + layer
+struct alignas(16) LayerScratch {  // private to the layer warp of a CTA
+    unsigned long long keys[1024 + 2];         // staged candidate keys, then the keys of R + layer
     unsigned long long lkeys[kMaxN];           // keys of the new layer, slot order
     double vals[kMaxN];                        // path values of the new running top-n
-    int toks[1024];                            // staged candidate tokens
+    int toks[1024 + 4];                        // staged candidate tokens
     int gids[2 * kMaxN];
     int rsel[kMaxN];                           // gids of the new running top-n, ascending
     int ltok[kMaxN];                           // tokens of the new layer, slot order
+    int mpos[kMaxN];                           // mailbox positions reserved for the new layer's rows
     int hist[256];
 };
 

@@ -108,7 +108,7 @@ __device__ int warp_compact_selected(KeyFn keyf, int N, unsigned long long thr, 
 
 // Per-sequence state and arrays in the workspace (device pointers already offset to the sequence).
 struct SeqWork {
-    double* cand_phat;     // [n*k]    path values of this layer's candidates (Eq. 2), slot-major
+    double* cand_phat;     // [n*k, padded to a multiple of 4, 16-byte aligned]  path values of this layer's candidates (Eq. 2), slot-major
     int32_t* cand_tok;     // [n*k]
     int32_t* T_tok;        // [D*n]    drafted nodes, gid = (depth-1)*n + slot
     int32_t* T_par;        // [D*n]    slot of the parent in the previous layer
@@ -130,7 +130,7 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
 // Layer job, first half.  After all rows of layer d (1-based) of one sequence are expanded: the
 // next layer = the nl candidates of largest path value, stored in candidate-index order (nodes
 // gid0 .. gid0+nl of T; tokens and keys also left in s.ltok / s.lkeys).  Whole layer warp; s is its scratch; fsize = rows of the layer.  Returns nl.
-__device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int fsize, int n, int k, int kk) {
+__device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int fsize, int n, int k, int kk, int* status) {
     const int lane = threadIdx.x & 31;
     int* hist = s.hist;
     const int N = fsize * k;
@@ -139,17 +139,46 @@ __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int f
     const int gid0 = (d - 1) * n;
     unsigned long long thr;
     int need_eq;
-    auto gkey = [&](int i) -> unsigned long long { return (i % k) < kk ? phat_key(__ldcg(&w.cand_phat[i])) : 0ull; };
+    // Candidate words validate themselves (written by other SMs' finisher warps without a fence): top
+    // bit set = written; all ones = no such child.  A word not yet written is simply read again.
+    const unsigned long long* gph = reinterpret_cast<const unsigned long long*>(w.cand_phat);
+    const unsigned int* gtk = reinterpret_cast<const unsigned int*>(w.cand_tok);
+    auto wait_phat = [&](int i) -> unsigned long long {
+        unsigned long long x = ld_relaxed_u64(&gph[i]);
+        for (int t = 0; !(x >> 63) && t < (1 << 22); ++t) x = ld_relaxed_u64(&gph[i]);
+        if (!(x >> 63)) { set_status(status, kErrTimeout); x = ~0ull; }
+        return x;
+    };
+    auto wait_tok = [&](int i) -> int {
+        unsigned int x = ld_relaxed_u32(&gtk[i]);
+        for (int t = 0; !(x >> 31) && t < (1 << 22); ++t) x = ld_relaxed_u32(&gtk[i]);
+        if (!(x >> 31)) { set_status(status, kErrTimeout); x = ~0u; }
+        return x == ~0u ? -1 : (int)(x & 0x7FFFFFFFu);
+    };
+    auto key_of = [](unsigned long long x) -> unsigned long long { return x == ~0ull ? 0ull : (x & 0x7FFFFFFFFFFFFFFFull) + 1ull; };
     unsigned long long ko = 0ull, ka = ~0ull;
-    if (N <= 1024) {                                      // stage keys and tokens in shared memory
-#pragma unroll 4
+    if (N <= 1024) {
+        // Stage path values and tokens in shared memory with 16-byte asynchronous copies, so that all
+        // loads are in flight together (one round trip); then the keys in place.  The per-sequence
+        // candidate arrays are padded to a multiple of four entries, so reading the last vector whole
+        // stays inside them.
+        for (int i = lane * 2; i < N; i += 64) cp_async_16(&s.keys[i], &gph[i]);
+        for (int i = lane * 4; i < N; i += 128) cp_async_16(&s.toks[i], &gtk[i]);
+        cp_async_wait_all();
+        __syncwarp();
         for (int i = lane; i < N; i += 32) {
-            const unsigned long long key = gkey(i);
+            unsigned long long x = s.keys[i];
+            if (!(x >> 63)) x = wait_phat(i);
+            const unsigned int t = (unsigned int)s.toks[i];
+            s.toks[i] = (t >> 31) ? (t == ~0u ? -1 : (int)(t & 0x7FFFFFFFu)) : wait_tok(i);
+            const unsigned long long key = key_of(x);
             s.keys[i] = key;
-            s.toks[i] = __ldcg(&w.cand_tok[i]);
             if (key) { ko |= key; ka &= key; }
         }
         __syncwarp();
+        // the arrays are free for the next layer's rows once they are zero again
+        for (int i = lane * 2; i < N; i += 64) *reinterpret_cast<uint4*>(&w.cand_phat[i]) = make_uint4(0, 0, 0, 0);
+        for (int i = lane * 4; i < N; i += 128) *reinterpret_cast<uint4*>(&w.cand_tok[i]) = make_uint4(0, 0, 0, 0);
         auto skey = [&](int i) -> unsigned long long { return s.keys[i]; };
         warp_radix_select(skey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
         warp_compact_selected(skey, N, thr, need_eq, [&](int pos, int i) {
@@ -160,6 +189,7 @@ __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int f
             s.lkeys[pos] = s.keys[i];
         });
     } else {
+        auto gkey = [&](int i) -> unsigned long long { return key_of(wait_phat(i)); };
         for (int i = lane; i < N; i += 32) {
             const unsigned long long key = gkey(i);
             if (key) { ko |= key; ka &= key; }
@@ -167,13 +197,16 @@ __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int f
         warp_radix_select(gkey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
         warp_compact_selected(gkey, N, thr, need_eq, [&](int pos, int i) {
             const unsigned long long key = gkey(i);
-            const int tok = __ldcg(&w.cand_tok[i]);
+            const int tok = wait_tok(i);
             w.T_tok[gid0 + pos] = tok;
             s.ltok[pos] = tok;
             w.T_par[gid0 + pos] = i / k;
             w.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
             s.lkeys[pos] = key;
         });
+        __syncwarp();
+        for (int i = lane * 2; i < N; i += 64) *reinterpret_cast<uint4*>(&w.cand_phat[i]) = make_uint4(0, 0, 0, 0);
+        for (int i = lane * 4; i < N; i += 128) *reinterpret_cast<uint4*>(&w.cand_tok[i]) = make_uint4(0, 0, 0, 0);
     }
     __syncwarp();
     return nl;
