@@ -8,18 +8,22 @@
 namespace ot {
 
 // CTA shape of the row pipeline (one CTA per SM): 16 consumer warps stream the logits, an issuer
-// warp feeds the shared-memory ring, a fetcher warp obtains row descriptors ahead of time, and
-// several finisher warps (one row each, round robin) turn finished rows into probabilities and
-// tree updates.  A lone warp advances slowly next to 16 busy ones, hence several finishers.  One
-// more warp takes whole-layer jobs of the tree build (selection of the next layer) from a queue.
+// warp feeds the shared-memory ring, a fetcher warp obtains row descriptors ahead of time, several
+// finisher warps (one row each, round robin) turn finished rows into probabilities and tree
+// updates, and a layer warp selects the next layer of the trees it follows.
+//
+// Warp w of a CTA issues from scheduler w % 4 of its SM.  The consumer warps have so much
+// independent work that a lone, dependent instruction stream next to them advances very slowly, so
+// the helper warps get a scheduler to themselves: warps with w % 4 == 3 are helpers, the others are
+// consumers (the first 16 of them; the rest of the 28 warps exit at once).
 constexpr int kConsumerWarps = 16;
 constexpr int kConsumers = kConsumerWarps * 32;     // 512 consumer threads
-constexpr int kIssuerWarp = kConsumerWarps;         // warp 16
-constexpr int kFetcherWarp = kConsumerWarps + 1;    // warp 17
-constexpr int kFirstFinisherWarp = kConsumerWarps + 2;
-constexpr int kFinishers = 6;
-constexpr int kLayerWarp = kFirstFinisherWarp + kFinishers;
-constexpr int kThreads = (kLayerWarp + 1) * 32;     // 800 threads per CTA
+constexpr int kFinishers = 4;
+constexpr int kHelperWarps = 3 + kFinishers;        // issuer, fetcher, layer warp, finishers
+constexpr int kWarps = 4 * kHelperWarps;            // 28: helper h is warp 4*h + 3
+constexpr int kThreads = kWarps * 32;               // 896 threads per CTA
+static_assert(kWarps - kHelperWarps >= kConsumerWarps, "not enough non-helper warps for the consumers");
+enum { kHelperIssuer = 0, kHelperFetcher = 1, kHelperLayer = 2, kHelperFirstFinisher = 3 };
 constexpr int kMaxK = 32;
 constexpr int kMaxN = 256;
 

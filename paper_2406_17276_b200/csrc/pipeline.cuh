@@ -133,8 +133,8 @@ __device__ void issuer_role(CtaSmem& s, int V, bool aligned, int* status) {
 }
 
 // ---- consumer warps ----------------------------------------------------------------------------
-__device__ void consumer_role(CtaSmem& s, int V, int* status) {
-    const int tid = threadIdx.x, lane = tid & 31;
+__device__ void consumer_role(CtaSmem& s, int cwarp, int V, int* status) {
+    const int lane = threadIdx.x & 31, tid = cwarp * 32 + lane;     // index among the consumer threads
     const int nchunks = (V + kChunkElems - 1) / kChunkElems;
     long long g = 0;
     ThreadAcc acc;
@@ -207,11 +207,16 @@ template <class Source, class Sink>
 __device__ __forceinline__ void run_pipeline(CtaSmem& s, Source& src, Sink& sink, int V, int k, bool aligned, int* status) {
     pipeline_init(s);
     const int warp = threadIdx.x >> 5;
-    if (warp < kConsumerWarps) consumer_role(s, V, status);
-    else if (warp == kIssuerWarp) issuer_role(s, V, aligned, status);
-    else if (warp == kFetcherWarp) fetcher_role(s, src, status);
-    else if (warp == kLayerWarp) sink.layer_loop(s.layer);
-    else finisher_role(s, sink, warp - kFirstFinisherWarp, V, k, aligned, status);
+    if ((warp & 3) != 3) {
+        const int cwarp = (warp >> 2) * 3 + (warp & 3);
+        if (cwarp < kConsumerWarps) consumer_role(s, cwarp, V, status);
+        return;
+    }
+    const int helper = warp >> 2;
+    if (helper == kHelperIssuer) issuer_role(s, V, aligned, status);
+    else if (helper == kHelperFetcher) fetcher_role(s, src, status);
+    else if (helper == kHelperLayer) sink.layer_loop(s.layer);
+    else finisher_role(s, sink, helper - kHelperFirstFinisher, V, k, aligned, status);
 }
 
 }  // namespace ot
