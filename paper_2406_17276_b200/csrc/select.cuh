@@ -106,6 +106,42 @@ __device__ int warp_compact_selected(KeyFn keyf, int N, unsigned long long thr, 
     return taken;
 }
 
+// The same selection, but every lane owns a contiguous stretch of `per` elements (lane l: indices
+// l*per .. l*per+per, cut at N), so that positions follow from one count per lane and one warp scan
+// instead of a ballot per 32 elements.  The kept indices go to idx[0..kept) first (a lane may own
+// many of them), then emit(pos, i) runs over the positions spread evenly over the lanes.  Returns
+// the number kept.  Whole warp.
+template <class KeyFn, class EmitFn>
+__device__ int warp_compact_selected_blocked(KeyFn keyf, int N, unsigned long long thr, int need_eq, int* idx, EmitFn emit) {
+    const int lane = threadIdx.x & 31;
+    const int per = (N + 31) >> 5;
+    const int lo = min(lane * per, N), hi = min(lo + per, N);
+    int gt = 0, eq = 0;
+#pragma unroll 4
+    for (int i = lo; i < hi; ++i) {
+        const unsigned long long key = keyf(i);
+        gt += key > thr ? 1 : 0;
+        eq += key == thr ? 1 : 0;
+    }
+    int total_eq, total;
+    const int eq_before = warp_excl_scan(eq, total_eq);
+    int eq_take = need_eq - eq_before;
+    eq_take = eq_take < 0 ? 0 : (eq_take > eq ? eq : eq_take);
+    int pos = warp_excl_scan(gt + eq_take, total);
+    if (gt + eq_take > 0) {
+        for (int i = lo; i < hi; ++i) {
+            const unsigned long long key = keyf(i);
+            bool take = key > thr;
+            if (key == thr && eq_take > 0) { take = true; --eq_take; }
+            if (take) idx[pos++] = i;
+        }
+    }
+    __syncwarp();
+    for (int q = lane; q < total; q += 32) emit(q, idx[q]);
+    __syncwarp();
+    return total;
+}
+
 // Per-sequence state and arrays in the workspace (device pointers already offset to the sequence).
 struct SeqWork {
     double* cand_phat;     // [n*k, padded to a multiple of 4, 16-byte aligned]  path values of this layer's candidates (Eq. 2), slot-major
@@ -166,11 +202,10 @@ __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int f
         for (int i = lane * 4; i < N; i += 128) cp_async_16(&s.toks[i], &gtk[i]);
         cp_async_wait_all();
         __syncwarp();
+#pragma unroll 4
         for (int i = lane; i < N; i += 32) {
             unsigned long long x = s.keys[i];
             if (!(x >> 63)) x = wait_phat(i);
-            const unsigned int t = (unsigned int)s.toks[i];
-            s.toks[i] = (t >> 31) ? (t == ~0u ? -1 : (int)(t & 0x7FFFFFFFu)) : wait_tok(i);
             const unsigned long long key = key_of(x);
             s.keys[i] = key;
             if (key) { ko |= key; ka &= key; }
@@ -181,9 +216,11 @@ __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int f
         for (int i = lane * 4; i < N; i += 128) *reinterpret_cast<uint4*>(&w.cand_tok[i]) = make_uint4(0, 0, 0, 0);
         auto skey = [&](int i) -> unsigned long long { return s.keys[i]; };
         warp_radix_select(skey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
-        warp_compact_selected(skey, N, thr, need_eq, [&](int pos, int i) {
-            w.T_tok[gid0 + pos] = s.toks[i];
-            s.ltok[pos] = s.toks[i];
+        warp_compact_selected_blocked(skey, N, thr, need_eq, s.gids, [&](int pos, int i) {
+            const unsigned int t = (unsigned int)s.toks[i];                  // staged word: top bit = written
+            const int tok = (t >> 31) ? (int)(t & 0x7FFFFFFFu) : wait_tok(i);
+            w.T_tok[gid0 + pos] = tok;
+            s.ltok[pos] = tok;
             w.T_par[gid0 + pos] = i / k;
             w.T_phat[gid0 + pos] = __longlong_as_double((long long)(s.keys[i] - 1ull));
             s.lkeys[pos] = s.keys[i];
