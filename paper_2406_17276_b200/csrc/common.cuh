@@ -12,16 +12,20 @@ namespace ot {
 // finisher warps (one row each, round robin) turn finished rows into probabilities and tree
 // updates, and a layer warp selects the next layer of the trees it follows.
 //
-// Warp w of a CTA issues from scheduler w % 4 of its SM.  The consumer warps have so much
-// independent work that a lone, dependent instruction stream next to them advances very slowly, so
-// the helper warps get a scheduler to themselves: warps with w % 4 == 3 are helpers, the others are
-// consumers (the first 16 of them; the rest of the 28 warps exit at once).
+// Warp w of a CTA issues from scheduler w % 4 of its SM.  With kPartition the helper warps get a
+// scheduler to themselves (warps with w % 4 == 3; the first 16 other warps are the consumers, the
+// rest exit at once): helpers then advance faster, consumers lose a quarter of the machine.
+// Without it the consumers are warps 0..15 and the helpers follow.
+#ifndef OT_PARTITION
+#define OT_PARTITION 0
+#endif
+constexpr bool kPartition = OT_PARTITION != 0;
 constexpr int kConsumerWarps = 16;
 constexpr int kConsumers = kConsumerWarps * 32;     // 512 consumer threads
-constexpr int kFinishers = 4;
+constexpr int kFinishers = kPartition ? 4 : 6;
 constexpr int kHelperWarps = 3 + kFinishers;        // issuer, fetcher, layer warp, finishers
-constexpr int kWarps = 4 * kHelperWarps;            // 28: helper h is warp 4*h + 3
-constexpr int kThreads = kWarps * 32;               // 896 threads per CTA
+constexpr int kWarps = kPartition ? 4 * kHelperWarps : kConsumerWarps + kHelperWarps;
+constexpr int kThreads = kWarps * 32;               // 896 / 800 threads per CTA
 static_assert(kWarps - kHelperWarps >= kConsumerWarps, "not enough non-helper warps for the consumers");
 enum { kHelperIssuer = 0, kHelperFetcher = 1, kHelperLayer = 2, kHelperFirstFinisher = 3 };
 constexpr int kMaxK = 32;

@@ -207,12 +207,18 @@ template <class Source, class Sink>
 __device__ __forceinline__ void run_pipeline(CtaSmem& s, Source& src, Sink& sink, int V, int k, bool aligned, int* status) {
     pipeline_init(s);
     const int warp = threadIdx.x >> 5;
-    if ((warp & 3) != 3) {
-        const int cwarp = (warp >> 2) * 3 + (warp & 3);
-        if (cwarp < kConsumerWarps) consumer_role(s, cwarp, V, status);
-        return;
+    int helper;
+    if (kPartition) {
+        if ((warp & 3) != 3) {
+            const int cwarp = (warp >> 2) * 3 + (warp & 3);
+            if (cwarp < kConsumerWarps) consumer_role(s, cwarp, V, status);
+            return;
+        }
+        helper = warp >> 2;
+    } else {
+        if (warp < kConsumerWarps) { consumer_role(s, warp, V, status); return; }
+        helper = warp - kConsumerWarps;
     }
-    const int helper = warp >> 2;
     if (helper == kHelperIssuer) issuer_role(s, V, aligned, status);
     else if (helper == kHelperFetcher) fetcher_role(s, src, status);
     else if (helper == kHelperLayer) sink.layer_loop(s.layer);
