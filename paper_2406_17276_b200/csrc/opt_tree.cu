@@ -319,7 +319,7 @@ struct BuildSink {
 
 // Algorithm 1 for a whole batch in one launch: persistent CTAs pull rows from the queue; layers
 // of different sequences overlap freely because sequences never exchange data.
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads)
 build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, opt_tree_out out) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
@@ -353,7 +353,7 @@ struct ListSink {
         }
     }
 };
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads)
 row_topk_kernel(Params p, const uint16_t* __restrict__ logits, const int32_t* __restrict__ rows, int nrows,
                 int32_t* tok_out, double* prob_out, int* status) {
     extern __shared__ __align__(128) unsigned char smem_raw[];

@@ -74,7 +74,7 @@ __device__ void fetcher_role(CtaSmem& s, Source& src, int* status) {
         const unsigned rm = __ballot_sync(0xFFFFFFFFu, got > 0), em = __ballot_sync(0xFFFFFFFFu, got < 0);
         if (got > 0) {
             const int a = known + __popc(rm & below);
-            s.desc[a % kDesc] = dsc;
+            s.desc[a % kDescRing] = dsc;
             mbar_arrive(&s.desc_full[a % kDesc]);              // release: publishes the descriptor
             holding = false;
         }
@@ -82,7 +82,7 @@ __device__ void fetcher_role(CtaSmem& s, Source& src, int* status) {
         if (em) {                                              // no more work: one stop marker after the last row
             if (lane == __ffs(em) - 1) {
                 dsc.stop = 1;
-                s.desc[known % kDesc] = dsc;
+                s.desc[known % kDescRing] = dsc;
                 mbar_arrive(&s.desc_full[known % kDesc]);
             }
             return;
@@ -105,8 +105,8 @@ __device__ void issuer_role(CtaSmem& s, int V, bool aligned, int* status) {
     for (int r = 0;; ++r) {
         const int e = r % kDesc;
         if (!mbar_wait_warp(&s.desc_full[e], (uint32_t)(r / kDesc) & 1u, status)) return;
-        const uint16_t* row = s.desc[e].row;
-        const int go = s.desc[e].stop ? 0 : 1;
+        const uint16_t* row = s.desc[r % kDescRing].row;
+        const int go = s.desc[r % kDescRing].stop ? 0 : 1;
         const int nc = go ? nchunks : 1;                       // the stop marker takes one (empty) chunk slot
         for (int c = 0; c < nc; ++c, ++g) {
             const int st = (int)(g % kStages);
@@ -133,40 +133,42 @@ __device__ void issuer_role(CtaSmem& s, int V, bool aligned, int* status) {
 }
 
 // ---- consumer warps ----------------------------------------------------------------------------
+// A warp takes its share of a chunk out of the ring into registers and hands the stage back at once
+// (so the issuer can refill it while the exponentials run); a row's descriptor is only looked at for
+// its stop flag.
 __device__ void consumer_role(CtaSmem& s, int cwarp, int V, int* status) {
     const int lane = threadIdx.x & 31, tid = cwarp * 32 + lane;     // index among the consumer threads
     const int nchunks = (V + kChunkElems - 1) / kChunkElems;
-    long long g = 0;
     ThreadAcc acc;
+    acc.reset();
+    ChunkRegs ch;
+    long long g = 0;
     for (int r = 0;; ++r) {
-        const int e = r % kDesc;
-        acc.reset();
-        RowDesc dsc;
         for (int c = 0; c < nchunks; ++c, ++g) {
             const int st = (int)(g % kStages);
             if (!mbar_wait_warp(&s.full_bar[st], (uint32_t)(g / kStages) & 1u, status)) return;
             if (c == 0) {
-                dsc = s.desc[e];
-                if (dsc.stop) break;
+                if (s.desc[r % kDescRing].stop) {
+                    if (tid == 0) s.stop_row = r;                  // the finishers poll this
+                    return;
+                }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&s.desc_empty[e]);  // this warp has its copy of the descriptor
+                if (lane == 0) mbar_arrive(&s.desc_empty[r % kDesc]);      // this warp has looked at the descriptor
             }
-            chunk_pass(acc, reinterpret_cast<const uint4*>(&s.stage[st][0]), (chunk_elems(V, c) + 7) >> 3, tid);
+            chunk_take(ch, reinterpret_cast<const uint4*>(&s.stage[st][0]), (chunk_elems(V, c) + 7) >> 3, tid);
             __syncwarp();
-            if (lane == 0) mbar_arrive(&s.empty_bar[st]);
-        }
-        if (dsc.stop) {
-            if (tid == 0) s.stop_row = r;                      // the finishers poll this
-            return;
+            if (lane == 0) mbar_arrive(&s.empty_bar[st]);          // the data is in registers: the stage is free
+            chunk_chain(ch);
+            const unsigned long long C2 = chunk_apply(acc, ch);
+            chunk_exps(acc, ch, C2);
         }
         // hand the row to its finisher
         const int sl = r % kSlots;
-        RowSlot& slot = s.slot[sl];
         if (r >= kSlots && !mbar_wait_warp(&s.free_bar[sl], (uint32_t)((r / kSlots) - 1) & 1u, status)) return;
-        store_thread_result(slot, acc, tid);
-        if (tid == 0) slot.desc = dsc;
+        store_thread_result(s.slot[sl], acc, tid);
         __syncwarp();
         if (lane == 0) mbar_arrive(&s.ready_bar[sl]);
+        acc.reset();
     }
 }
 
@@ -194,9 +196,9 @@ __device__ void finisher_role(CtaSmem& s, Sink& sink, int fidx, int V, int k, bo
             if (!__all_sync(0xFFFFFFFFu, ok)) return;
         }
         const RowSlot& slot = s.slot[sl];
+        const RowDesc dsc = s.desc[r % kDescRing];
         RowOut out;
-        finish_row_warp(f, slot, V, k, aligned, out);
-        const RowDesc dsc = slot.desc;
+        finish_row_warp(f, slot, dsc.row, V, k, aligned, out);
         __syncwarp();
         if (lane == 0) mbar_arrive(&s.free_bar[sl]);                              // the slot can be refilled
         sink.row_done(dsc, out, f);

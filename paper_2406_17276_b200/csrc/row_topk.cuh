@@ -34,6 +34,7 @@ constexpr int kSlots = kFinishers + 2;             // finished rows waiting for 
 constexpr int kCandCap = 128;                      // candidate list capacity per row
 constexpr int kMaxFlag = 64;                       // flagged threads the fast finisher accepts
 constexpr int kDesc = 4;                           // rows a CTA may hold between ticket and descriptor read
+constexpr int kDescRing = 16;                      // descriptors kept: a row's lives until its finisher has copied it
 constexpr int kPerLane = kConsumers / 32;          // per-thread results one finisher lane handles (16)
 
 constexpr float kLog2e = 1.44269504088896340736f;
@@ -58,7 +59,6 @@ struct alignas(16) RowSlot {
     float tsum[kConsumers];
     uint16_t tkey[kConsumers];     // per-thread maximum as an ordered key
     int warpE[kConsumerWarps];
-    RowDesc desc;
 };
 
 struct FinScratch {                // private to one finisher warp
@@ -81,13 +81,15 @@ struct alignas(16) LayerScratch {  // private to the layer warp of a CTA
 };
 
 static_assert(sizeof(RowSlot) % 16 == 0, "slots must keep 16-byte alignment in an array");
+// rows between "descriptor written" and "finisher has its copy": kDesc known + 1 streaming + kSlots handed on
+static_assert(kDescRing >= kDesc + 1 + kSlots + 1, "descriptor ring too short");
 
 struct alignas(128) CtaSmem {
     uint16_t stage[kStages][kChunkElems];
     RowSlot slot[kSlots];
     FinScratch fin[kFinishers];
     LayerScratch layer;
-    RowDesc desc[kDesc];
+    RowDesc desc[kDescRing];                   // row r in entry r % kDescRing
     unsigned long long full_bar[kStages];      // issuer -> consumers (bulk copy landed)
     unsigned long long empty_bar[kStages];     // consumers -> issuer (stage may be overwritten)
     unsigned long long ready_bar[kSlots];      // consumers -> finisher (slot filled)
@@ -116,33 +118,55 @@ __device__ __forceinline__ float pow2_float(int d) {            // 2^d for d <= 
     return __int_as_float(max(d + 127, 0) << 23);
 }
 
-// This thread's share of one chunk (kVecPerThread vectors of 8 logits) folded into its state.
-__device__ __forceinline__ void chunk_pass(ThreadAcc& a, const uint4* vec, int nv, int tid) {
+// One chunk's share of a consumer thread, taken out of the ring into registers: kVecPerThread
+// vectors of 8 logits, their packed maximum and the integer exponent that maximum asks for.
+struct ChunkRegs {
     uint4 w[kVecPerThread];
+    uint32_t m2;
+    float Ec;
+};
+
+__device__ __forceinline__ void chunk_take(ChunkRegs& c, const uint4* vec, int nv, int tid) {
 #pragma unroll
     for (int u = 0; u < kVecPerThread; ++u) {
         const int v = tid + u * kConsumers;
-        w[u] = v < nv ? vec[v] : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // -inf padding
+        c.w[u] = v < nv ? vec[v] : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // -inf padding
     }
-    // maximum of the 32 logits, then the exponent they are summed against
+}
+
+// Maximum of the 32 logits and the exponent they want to be summed against (any integer >= max*log2e
+// will do: the magic-number add rounds max*log2e + 1 to the nearest integer on the FMA pipe).
+__device__ __forceinline__ void chunk_chain(ChunkRegs& c) {
     uint32_t m2 = 0xFF80FF80u;
 #pragma unroll
     for (int u = 0; u < kVecPerThread; ++u)
-        m2 = max_bf16x2(m2, max_bf16x2(max_bf16x2(w[u].x, w[u].y), max_bf16x2(w[u].z, w[u].w)));
-    a.pm = max_bf16x2(a.pm, m2);
+        m2 = max_bf16x2(m2, max_bf16x2(max_bf16x2(c.w[u].x, c.w[u].y), max_bf16x2(c.w[u].z, c.w[u].w)));
+    c.m2 = m2;
     const float f = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
-    float Ec;
-    asm("cvt.rpi.f32.f32 %0, %1;" : "=f"(Ec) : "f"(fminf(fmaxf(f * kLog2e, kExpFloor), -kExpFloor)));
-    const float En = fmaxf(a.E, Ec);
-    const float sc = pow2_float((int)(a.E - En));                    // exact: both are integers
+    const float t = fminf(fmaxf(fmaf(f, kLog2e, 1.0f), kExpFloor), -kExpFloor);
+    c.Ec = (t + 12582912.0f) - 12582912.0f;
+}
+
+// Folds the chunk's maximum into the thread's state (raising E rescales the sums by an exact power
+// of two) and returns the packed constant -E for the exponentials.
+__device__ __forceinline__ unsigned long long chunk_apply(ThreadAcc& a, const ChunkRegs& c) {
+    a.pm = max_bf16x2(a.pm, c.m2);
+    const float En = fmaxf(a.E, c.Ec);
+    const int d = __float_as_int((a.E - En) + 12582912.0f) - 0x4B400000;     // a.E - En as an integer (<= 0, exact)
+    const float sc = pow2_float(d);
     const unsigned long long sc2 = pack2(sc, sc);
     a.acc0 = mul2(a.acc0, sc2);
     a.acc1 = mul2(a.acc1, sc2);
     a.E = En;
-    const unsigned long long L2 = pack2(kLog2e, kLog2e), C2 = pack2(-En, -En);
+    return pack2(-En, -En);
+}
+
+// The 32 exponentials of a chunk: 2^(x*log2e - E) in packed fp32x2 FMA + ex2.approx.
+__device__ __forceinline__ void chunk_exps(ThreadAcc& a, const ChunkRegs& c, unsigned long long C2) {
+    const unsigned long long L2 = pack2(kLog2e, kLog2e);
 #pragma unroll
     for (int u = 0; u < kVecPerThread; ++u) {
-        const uint32_t ww[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+        const uint32_t ww[4] = {c.w[u].x, c.w[u].y, c.w[u].z, c.w[u].w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const float lo = __uint_as_float(ww[i] << 16), hi = __uint_as_float(ww[i] & 0xFFFF0000u);
@@ -345,7 +369,7 @@ __device__ __forceinline__ uint4 load_row_vec(const uint16_t* row, int vi, int V
 }
 
 // Turns a finished slot into the row's k winners.  Whole finisher warp; f is its private scratch.
-__device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& slot, int V, int k, bool aligned, RowOut& out) {
+__device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& slot, const uint16_t* row, int V, int k, bool aligned, RowOut& out) {
     const int lane = threadIdx.x & 31;
     const int kk = k < V ? k : V;
     const int nvec = (V + 7) >> 3;
@@ -462,7 +486,7 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
                 if (idx < total) {
                     const int fi = idx / vpt, j = idx - fi * vpt;
                     const int vi = (j / kVecPerThread) * kChunkVecs + (j % kVecPerThread) * kConsumers + f.flist[fi];
-                    if (vi < nvec) { vis[u] = vi; w[u] = load_row_vec(slot.desc.row, vi, V, aligned); }
+                    if (vi < nvec) { vis[u] = vi; w[u] = load_row_vec(row, vi, V, aligned); }
                 }
             }
 #pragma unroll
@@ -493,7 +517,7 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
         }
     }
     if (exact) {
-        row_exact_warp(f, slot.desc.row, V, kk, m, S);
+        row_exact_warp(f, row, V, kk, m, S);
         M = f.cand_count;                                     // == kk <= 32
     }
     __syncwarp();
