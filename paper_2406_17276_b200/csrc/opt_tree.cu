@@ -231,13 +231,15 @@ struct BuildSink {
         __syncwarp();
         if (lane == 0) atom_add_relaxed_s32(&sw.st[kStDone], 1);     // the count runs on over the layers of a build
     }
-    // Rows of layer d+1 of sequence b go to consecutive CTAs starting at a CTA that depends on (b, d),
-    // so that one layer spreads over as many SMs as it has rows.  reserve_layer takes their mailbox
+    // Rows of layer d+1 of sequence b go to consecutive CTAs, so that one layer spreads over as many
+    // SMs as it has rows.  Sequence b starts where sequence b-1's rows of an equally large layer end:
+    // the layers of all sequences then tile the CTAs evenly (a start that ignores the layer's size
+    // gives some CTAs twice the rows of others); the layer index only rotates the tiling.  reserve_layer takes their mailbox
     // positions (into ls.mpos), publish_layer writes the entries once the nodes are chosen.
-    __device__ int first_cta(int b, int d) const { return (int)(((unsigned)b * 37u + (unsigned)d * 61u) % (unsigned)p.grid); }
+    __device__ int first_cta(int b, int d, int nl) const { return (int)(((unsigned)b * (unsigned)nl + (unsigned)d * 61u) % (unsigned)p.grid); }
     __device__ void reserve_layer(LayerScratch& ls, int b, int d, int nl) {
         const int lane = threadIdx.x & 31;
-        const int c0 = first_cta(b, d);
+        const int c0 = first_cta(b, d, nl);
         for (int i = lane; i < nl; i += 32) {
             const int c = (c0 + i) % p.grid;
             ls.mpos[i] = c * p.mcap + atomicAdd(&w.mb_tail[c], 1);
@@ -246,7 +248,7 @@ struct BuildSink {
     }
     __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl) {
         const int lane = threadIdx.x & 31;
-        const int c0 = first_cta(b, d);
+        const int c0 = first_cta(b, d, nl);
         for (int i = lane; i < nl; i += 32) {
             int token = ls.ltok[i];
             if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }

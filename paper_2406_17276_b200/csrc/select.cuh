@@ -209,6 +209,10 @@ __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int f
             const unsigned long long key = key_of(x);
             s.keys[i] = key;
             if (key) { ko |= key; ka &= key; }
+            // a token word that was not yet there when it was staged must be fetched before the arrays are
+            // cleared: a store that lands late would otherwise be wiped out, or wipe out a later layer's word
+            const unsigned int t = (unsigned int)s.toks[i];
+            if (!(t >> 31)) { const int tok = wait_tok(i); s.toks[i] = tok < 0 ? -1 : (int)(0x80000000u | (unsigned int)tok); }
         }
         __syncwarp();
         // the arrays are free for the next layer's rows once they are zero again
@@ -217,8 +221,8 @@ __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int f
         auto skey = [&](int i) -> unsigned long long { return s.keys[i]; };
         warp_radix_select(skey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
         warp_compact_selected_blocked(skey, N, thr, need_eq, s.gids, [&](int pos, int i) {
-            const unsigned int t = (unsigned int)s.toks[i];                  // staged word: top bit = written
-            const int tok = (t >> 31) ? (int)(t & 0x7FFFFFFFu) : wait_tok(i);
+            const unsigned int t = (unsigned int)s.toks[i];                  // staged word, validated above
+            const int tok = t == ~0u ? -1 : (int)(t & 0x7FFFFFFFu);
             w.T_tok[gid0 + pos] = tok;
             s.ltok[pos] = tok;
             w.T_par[gid0 + pos] = i / k;
