@@ -33,11 +33,12 @@ struct Workspace {
     int32_t* R;            // [B][2][n]
     double* E_prev;        // [B]
     int32_t* st;           // [B][8]
-    // row mailboxes of the build: one per CTA, filled by the layer warps, never wrapped within a build
+    // row mailboxes of the build: one per CTA, filled by the layer warps, never wrapped within a build.
+    // The rows of a build are numbered by one running count (q_ctl[kQCursor]): row g goes to CTA
+    // g % grid, entry g / grid of its mailbox.
     unsigned long long* mb_items;  // [grid][mcap]  one item per (sequence, layer, frontier slot)
     unsigned long long* mb_phat;   // [grid][mcap]  bit 63 valid | bits of the node's path value (a double >= 0)
-    int32_t* mb_tail;      // [grid]  entries reserved so far
-    int32_t* q_ctl;        // [8]  2: sequences finished, 3: all done
+    int32_t* q_ctl;        // [8]  2: sequences finished, 3: all done, 4: rows numbered so far
     // verify
     int32_t* g;            // [B][n+1]  target argmax after the root (0) and after node i (i+1)
     int32_t* vdone;        // [B]
@@ -49,16 +50,17 @@ struct Workspace {
     uint64_t* o_mask; int32_t* o_pos;
     int32_t *o_alen, *o_atok, *o_anode, *o_next;
 };
-enum { kQFinished = 2, kQDone = 3 };
+enum { kQFinished = 2, kQDone = 3, kQCursor = 4 };
 
 constexpr int kMaxGrid = 4096;              // CTAs of the persistent kernels (SMs x occupancy) this layout supports
 
-// Rows of one layer go to consecutive CTAs, so a CTA receives at most ceil(n / grid) rows per
-// (sequence, layer); its mailbox holds every row it can be sent during one build.
+// Consecutive rows go to consecutive CTAs, so a CTA receives its even share of all rows of a build
+// (one root and at most Dcap layers of n rows per sequence); its mailbox holds them all.
 static size_t mailbox_capacity(const opt_tree_config& c, int grid) {
     const size_t Dcap = c.max_depth < c.n ? c.max_depth : c.n;
+    const size_t rows = (size_t)c.max_batch * (1 + Dcap * (size_t)c.n);
     // + 8: a fetcher takes a few tickets beyond the last row it will ever get; those must stay inside
-    return (size_t)c.max_batch * Dcap * (((size_t)c.n + grid - 1) / grid) + 8;
+    return (rows + grid - 1) / grid + 8;
 }
 
 // Entries per sequence in the candidate arrays: n*k rounded up to a multiple of four (16-byte vectors).
@@ -89,7 +91,6 @@ static size_t carve(const opt_tree_config& c, int grid, char* base, Workspace* w
     OT_TAKE(st, int32_t, B * 8)
     OT_TAKE(mb_items, unsigned long long, mailbox_capacity(c, grid) * grid)
     OT_TAKE(mb_phat, unsigned long long, mailbox_capacity(c, grid) * grid)
-    OT_TAKE(mb_tail, int32_t, grid)
     OT_TAKE(q_ctl, int32_t, 8)
     OT_TAKE(g, int32_t, B * (n + 1))
     OT_TAKE(vdone, int32_t, B)
@@ -178,7 +179,6 @@ __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restri
         w.mb_items[i] = item;
         w.mb_phat[i] = ph;
     }
-    if (i < p.grid) w.mb_tail[i] = i < p.B ? (p.B - i + p.grid - 1) / p.grid : 0;
     for (long long j = i; j < (long long)p.B * p.cstride; j += (long long)gridDim.x * blockDim.x) {
         reinterpret_cast<unsigned long long*>(w.cand_phat)[j] = 0ull;
         w.cand_tok[j] = 0;
@@ -188,7 +188,7 @@ __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restri
         st[kStDone] = 0; st[kStNR] = 0;
         w.E_prev[i] = 0.0;
     }
-    if (i == 0) { w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; }
+    if (i == 0) { w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; w.q_ctl[kQCursor] = p.B; }   // the roots are rows 0 .. B-1
 }
 
 // Source of the tree build: the rows other CTAs' layer warps have put into this CTA's mailbox.
@@ -231,29 +231,25 @@ struct BuildSink {
         __syncwarp();
         if (lane == 0) atom_add_relaxed_s32(&sw.st[kStDone], 1);     // the count runs on over the layers of a build
     }
-    // Rows of layer d+1 of sequence b go to consecutive CTAs, so that one layer spreads over as many
-    // SMs as it has rows.  Sequence b starts where sequence b-1's rows of an equally large layer end:
-    // the layers of all sequences then tile the CTAs evenly (a start that ignores the layer's size
-    // gives some CTAs twice the rows of others); the layer index only rotates the tiling.  reserve_layer takes their mailbox
-    // positions (into ls.mpos), publish_layer writes the entries once the nodes are chosen.
-    __device__ int first_cta(int b, int d, int nl) const { return (int)(((unsigned)b * (unsigned)nl + (unsigned)d * 61u) % (unsigned)p.grid); }
-    __device__ void reserve_layer(LayerScratch& ls, int b, int d, int nl) {
-        const int lane = threadIdx.x & 31;
-        const int c0 = first_cta(b, d, nl);
-        for (int i = lane; i < nl; i += 32) {
-            const int c = (c0 + i) % p.grid;
-            ls.mpos[i] = c * p.mcap + atomicAdd(&w.mb_tail[c], 1);
-        }
-        __syncwarp();
+    // The rows of a new layer take the next numbers of the build's running row count and with them
+    // their CTAs (row g: CTA g % grid, mailbox entry g / grid).  Whatever the order in which the
+    // sequences publish, every CTA is sent the same number of rows to within one, and a layer spreads
+    // over as many SMs as it has rows.  reserve_layer only starts the atomic (lane 0 keeps the result
+    // in a register; nothing waits for it until publish_layer writes the entries).
+    __device__ unsigned reserve_layer(int nl) {
+        unsigned g0 = 0;
+        if ((threadIdx.x & 31) == 0) g0 = atomicAdd(reinterpret_cast<unsigned int*>(&w.q_ctl[kQCursor]), (unsigned)nl);
+        return g0;
     }
-    __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl) {
+    __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl, unsigned g0) {
         const int lane = threadIdx.x & 31;
-        const int c0 = first_cta(b, d, nl);
+        g0 = __shfl_sync(0xFFFFFFFFu, g0, 0);
         for (int i = lane; i < nl; i += 32) {
             int token = ls.ltok[i];
             if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
-            const int c = (c0 + i) % p.grid, pos = ls.mpos[i];
-            if (pos - c * p.mcap < p.mcap) {
+            const unsigned g = g0 + (unsigned)i, c = g % (unsigned)p.grid, e = g / (unsigned)p.grid;
+            if (e < (unsigned)p.mcap) {
+                const size_t pos = (size_t)c * p.mcap + e;
                 st_relaxed_u64(&w.mb_phat[pos], (1ull << 63) | (ls.lkeys[i] - 1ull));
                 st_relaxed_u64(&w.mb_items[pos], item_encode(b, d + 1, i, row_of(token, d, p.H)));
             } else {
@@ -292,14 +288,15 @@ struct BuildSink {
                     // Without a threshold the loop test only looks at the depth: the next layer's rows
                     // can go out before the running top-n is brought up to date.
                     const bool early = d < p.Dcap && p.delta == -INFINITY;
-                    if (early) reserve_layer(ls, b, d, nl);   // the mailbox positions, while the candidates load
+                    stage_layer_candidates(ls, sw, fsize, p.k);
+                    unsigned g0 = 0;
+                    if (early) g0 = reserve_layer(nl);        // the rows' numbers, while the candidates load
                     select_layer_warp(ls, sw, d, fsize, p.n, p.k, p.kk, w.status);
-                    if (early) publish_layer(ls, b, d, nl);
+                    if (early) publish_layer(ls, b, d, nl, g0);
                     const bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta,
                                                           w.status);
                     if (more && !early) {
-                        reserve_layer(ls, b, d, nl);
-                        publish_layer(ls, b, d, nl);
+                        publish_layer(ls, b, d, nl, reserve_layer(nl));
                     }
                     if (more) { cur_d[q] = d + 1; cur_f[q] = nl; cur_tot[q] += nl; }
                     else {

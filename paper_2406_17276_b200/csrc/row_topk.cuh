@@ -76,7 +76,6 @@ struct alignas(16) LayerScratch {  // private to the layer warp of a CTA
     int gids[2 * kMaxN];
     int rsel[kMaxN];                           // gids of the new running top-n, ascending
     int ltok[kMaxN];                           // tokens of the new layer, slot order
-    int mpos[kMaxN];                           // mailbox positions reserved for the new layer's rows
     int hist[256];
 };
 
@@ -435,7 +434,7 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
     }
     bool exact = tau_key <= kOrdNegInf || emax >= kExpLimit || emax <= -kExpLimit;
 
-    // bulk of the unflagged threads; flagged threads listed in thread order
+    // the sum of all threads' partial sums; flagged threads listed in thread order
     uint32_t fmask = 0;
     float part32 = 0.0f;
     {
@@ -443,13 +442,9 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
 #pragma unroll
         for (int q = 0; q < kPerLane / 4; ++q) {
             const float4 t4 = sp[q];
-            const float tt[4] = {t4.x, t4.y, t4.z, t4.w};
+            part32 += (t4.x + t4.y) + (t4.z + t4.w);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const bool fl = key[q * 4 + i] >= tau_key;
-                fmask |= fl ? (1u << (q * 4 + i)) : 0u;
-                part32 += fl ? 0.0f : tt[i];
-            }
+            for (int i = 0; i < 4; ++i) fmask |= key[q * 4 + i] >= tau_key ? (1u << (q * 4 + i)) : 0u;
         }
     }
     int nflag = 0;
@@ -469,13 +464,16 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
     int M = 0;
     if (!exact) {
         const double part = (double)(part32 * pow2_float(myE - emax));
-        // flagged threads: read their vectors again, split candidates from bulk
+        // Flagged threads: their vectors are read again only to find the candidates (logit >= tau) and
+        // their tokens.  A candidate's term is already inside its thread's partial sum; the same
+        // approximate term is taken out again here (the two differ by rounding of the exponent, a
+        // few 1e-8 of the term), and the candidate comes back below with an exact exponential.
         const float tau_f = bf16_bits_to_float(ord16_inv(tau_key));
         const int nchunks = (V + kChunkElems - 1) / kChunkElems;
         const int vpt = nchunks * kVecPerThread;
         const int total = nflag * vpt;
         const float negE = -(float)emax;
-        float fb = 0.0f;
+        float sub = 0.0f;
         for (int i0 = 0; i0 < total; i0 += 32 * 4) {
             uint4 w[4];
             int vis[4];
@@ -483,6 +481,7 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
             for (int u = 0; u < 4; ++u) {
                 const int idx = i0 + u * 32 + lane;
                 vis[u] = -1;
+                w[u] = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
                 if (idx < total) {
                     const int fi = idx / vpt, j = idx - fi * vpt;
                     const int vi = (j / kVecPerThread) * kChunkVecs + (j % kVecPerThread) * kConsumers + f.flist[fi];
@@ -491,7 +490,9 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                if (vis[u] < 0) continue;
+                const uint32_t m2 = max_bf16x2(max_bf16x2(w[u].x, w[u].y), max_bf16x2(w[u].z, w[u].w));
+                const float vm = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
+                if (vis[u] < 0 || !(vm >= tau_f)) continue;                       // most vectors hold no candidate
                 const uint32_t ww[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
@@ -500,8 +501,7 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
                     if (x >= tau_f) {
                         const int pos = atomicAdd(&f.cand_count, 1);
                         if (pos < kCandCap) f.cand[pos] = cand_key(bits, (uint32_t)(vis[u] * 8 + e));
-                    } else {
-                        fb += ex2_approx(fmaf(x, kLog2e, negE));
+                        sub += ex2_approx(fmaf(x, kLog2e, negE));
                     }
                 }
             }
@@ -513,7 +513,7 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
             // Bulk terms are 2^(fl(x*L32) - E) with L32 the fp32 log2(e); wanted e^(x-m) = 2^((x-m)*L).
             // The exponent gap E - m*L + x*(L - L32) is evaluated at a typical bulk logit x = tau - 2.
             const double gap = (double)emax - m * kLog2eD + ((double)tau_f - 2.0) * (kLog2eD - (double)kLog2e);
-            S = warp_sum(part + (double)fb) * exp2(gap);
+            S = warp_sum(part - (double)sub) * exp2(gap);
         }
     }
     if (exact) {

@@ -163,6 +163,19 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
     double* esub_trace;    // may be null
 };
 
+// Starts the asynchronous copies of a layer's candidates (path values and tokens) into the layer
+// warp's scratch; select_layer_warp waits for them.  Separate so that other round trips (the
+// mailbox reservations) can be in flight at the same time.
+__device__ __forceinline__ void stage_layer_candidates(LayerScratch& s, const SeqWork& w, int fsize, int k) {
+    const int lane = threadIdx.x & 31;
+    const int N = fsize * k;
+    if (N > 1024) return;
+    const unsigned long long* gph = reinterpret_cast<const unsigned long long*>(w.cand_phat);
+    const unsigned int* gtk = reinterpret_cast<const unsigned int*>(w.cand_tok);
+    for (int i = lane * 2; i < N; i += 64) cp_async_16(&s.keys[i], &gph[i]);
+    for (int i = lane * 4; i < N; i += 128) cp_async_16(&s.toks[i], &gtk[i]);
+}
+
 // Layer job, first half.  After all rows of layer d (1-based) of one sequence are expanded: the
 // next layer = the nl candidates of largest path value, stored in candidate-index order (nodes
 // gid0 .. gid0+nl of T; tokens and keys also left in s.ltok / s.lkeys).  Whole layer warp; s is its scratch; fsize = rows of the layer.  Returns nl.
@@ -198,8 +211,7 @@ __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int f
         // loads are in flight together (one round trip); then the keys in place.  The per-sequence
         // candidate arrays are padded to a multiple of four entries, so reading the last vector whole
         // stays inside them.
-        for (int i = lane * 2; i < N; i += 64) cp_async_16(&s.keys[i], &gph[i]);
-        for (int i = lane * 4; i < N; i += 128) cp_async_16(&s.toks[i], &gtk[i]);
+        // (the copies were started by stage_layer_candidates)
         cp_async_wait_all();
         __syncwarp();
 #pragma unroll 4
