@@ -10,24 +10,23 @@ namespace ot {
 // CTA shape of the row pipeline (one CTA per SM): 16 consumer warps stream the logits, an issuer
 // warp feeds the shared-memory ring, a fetcher warp obtains row descriptors ahead of time, several
 // finisher warps (one row each, round robin) turn finished rows into probabilities and tree
-// updates, and a layer warp selects the next layer of the trees it follows.
+// updates, and a layer team (the layer warp and its assistants) selects the next layer of the
+// trees the CTA follows.
 //
-// Warp w of a CTA issues from scheduler w % 4 of its SM.  With kPartition the helper warps get a
-// scheduler to themselves (warps with w % 4 == 3; the first 16 other warps are the consumers, the
-// rest exit at once): helpers then advance faster, consumers lose a quarter of the machine.
-// Without it the consumers are warps 0..15 and the helpers follow.
-#ifndef OT_PARTITION
-#define OT_PARTITION 0
-#endif
-constexpr bool kPartition = OT_PARTITION != 0;
+// Warp w of a CTA issues from scheduler w % 4 of its SM: the consumers are warps 0..15, the
+// helpers follow, ordered so that the four warps of the layer team sit on four different
+// schedulers.  (Helper warps advance at roughly half their speed while the consumers are busy,
+// which is why the layer selection, the longest serial step between two layers, is spread over
+// several of them.)
 constexpr int kConsumerWarps = 16;
 constexpr int kConsumers = kConsumerWarps * 32;     // 512 consumer threads
-constexpr int kFinishers = kPartition ? 4 : 6;
-constexpr int kHelperWarps = 3 + kFinishers;        // issuer, fetcher, layer warp, finishers
-constexpr int kWarps = kPartition ? 4 * kHelperWarps : kConsumerWarps + kHelperWarps;
-constexpr int kThreads = kWarps * 32;               // 896 / 800 threads per CTA
-static_assert(kWarps - kHelperWarps >= kConsumerWarps, "not enough non-helper warps for the consumers");
-enum { kHelperIssuer = 0, kHelperFetcher = 1, kHelperLayer = 2, kHelperFirstFinisher = 3 };
+constexpr int kFinishers = 6;
+constexpr int kTeamWarps = 4;                       // layer warp + assistants
+constexpr int kTeam = kTeamWarps * 32;
+constexpr int kHelperWarps = 2 + kTeamWarps + kFinishers;
+constexpr int kWarps = kConsumerWarps + kHelperWarps;
+constexpr int kThreads = kWarps * 32;               // 896 threads per CTA
+enum { kHelperIssuer = 0, kHelperFetcher = 1, kHelperLayer = 2, kHelperFirstAssistant = 3, kHelperFirstFinisher = 2 + kTeamWarps };
 constexpr int kMaxK = 32;
 constexpr int kMaxN = 256;
 
@@ -185,6 +184,9 @@ __device__ __forceinline__ bool mbar_wait_thread(unsigned long long* bar, uint32
     }
     return true;
 }
+
+// --- barrier of the layer team (named barrier 1; barrier 0 is the CTA's) ---
+__device__ __forceinline__ void team_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kTeam) : "memory"); }
 
 // --- asynchronous global -> shared copies (16 bytes, L2 only: the data was written by other SMs;
 //     all copies of a sweep are in flight at once and need no registers) ---

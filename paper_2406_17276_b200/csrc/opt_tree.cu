@@ -258,7 +258,25 @@ struct BuildSink {
         }
         __syncwarp();
     }
+    // The layer warp follows its sequences (layer_follow); whenever a layer is complete it hands the
+    // selection to the whole team: the job goes into shared memory, the team barrier starts it.  The
+    // assistants wait at that barrier in between and leave when they find a job of kind 0.
     __device__ void layer_loop(LayerScratch& ls) {
+        layer_follow(ls);
+        if ((threadIdx.x & 31) == 0) ls.job.kind = 0;
+        __syncwarp();
+        team_sync();
+    }
+    __device__ void layer_assist(LayerScratch& ls, int tw) {
+        const int tt = tw * 32 + (int)(threadIdx.x & 31);
+        for (;;) {
+            team_sync();
+            const LayerJob j = ls.job;
+            if (j.kind == 0) return;
+            select_layer_team(ls, j, tt, w.status);
+        }
+    }
+    __device__ void layer_follow(LayerScratch& ls) {
         const int lane = threadIdx.x & 31;
         constexpr int kOwn = 4;                            // sequences one layer warp follows at a time
         for (int b0 = blockIdx.x; b0 < p.B; b0 += kOwn * gridDim.x) {
@@ -291,7 +309,21 @@ struct BuildSink {
                     stage_layer_candidates(ls, sw, fsize, p.k);
                     unsigned g0 = 0;
                     if (early) g0 = reserve_layer(nl);        // the rows' numbers, while the candidates load
-                    select_layer_warp(ls, sw, d, fsize, p.n, p.k, p.kk, w.status);
+                    if (fsize * p.k <= 1024) {
+                        if (lane == 0) {
+                            LayerJob& j = ls.job;
+                            j.kind = 1; j.d = d; j.fsize = fsize; j.n = p.n; j.k = p.k; j.kk = p.kk;
+                            j.cand_phat = sw.cand_phat; j.cand_tok = sw.cand_tok;
+                            j.T_tok = sw.T_tok; j.T_par = sw.T_par; j.T_phat = sw.T_phat;
+                        }
+                        cp_async_wait_all();                  // the staged candidates are in shared memory
+                        __syncwarp();
+                        team_sync();                          // ... and, with the job, visible to the assistants
+                        const LayerJob j = ls.job;
+                        select_layer_team(ls, j, lane, w.status);
+                    } else {
+                        select_layer_warp(ls, sw, d, fsize, p.n, p.k, p.kk, w.status);
+                    }
                     if (early) publish_layer(ls, b, d, nl, g0);
                     const bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta,
                                                           w.status);
@@ -344,6 +376,7 @@ struct ListSource {
 struct ListSink {
     int32_t* tok_out; double* prob_out; int k;
     __device__ void layer_loop(LayerScratch&) {}
+    __device__ void layer_assist(LayerScratch&, int) {}
     __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch&) {
         const int lane = threadIdx.x & 31;
         if (lane < k) {

@@ -12,7 +12,8 @@
 //                   gives them to a Sink (for the tree build: candidates' path values and the
 //                   layer's row counter);
 //   layer warp      runs Sink::layer_loop (for the tree build: watches the row counters of its
-//                   sequences, selects each next layer and publishes its rows).
+//                   sequences, selects each next layer and publishes its rows); its assistants
+//                   run Sink::layer_assist and share the selection's work.
 //
 // The chunks of consecutive rows form one stream: chunk g lives in stage g % kStages and is the
 // (g / kStages)-th use of that stage, which fixes every mbarrier parity; likewise row r uses
@@ -33,6 +34,7 @@ __device__ __forceinline__ void pipeline_init(CtaSmem& s) {
         s.stop_row = 0x7FFFFFFF;
         mbar_fence_init();
     }
+    for (int i = threadIdx.x; i < 3 * 256; i += kThreads) (&s.layer.thist[0][0])[i] = 0;
     __syncthreads();
 }
 
@@ -209,21 +211,12 @@ template <class Source, class Sink>
 __device__ __forceinline__ void run_pipeline(CtaSmem& s, Source& src, Sink& sink, int V, int k, bool aligned, int* status) {
     pipeline_init(s);
     const int warp = threadIdx.x >> 5;
-    int helper;
-    if (kPartition) {
-        if ((warp & 3) != 3) {
-            const int cwarp = (warp >> 2) * 3 + (warp & 3);
-            if (cwarp < kConsumerWarps) consumer_role(s, cwarp, V, status);
-            return;
-        }
-        helper = warp >> 2;
-    } else {
-        if (warp < kConsumerWarps) { consumer_role(s, warp, V, status); return; }
-        helper = warp - kConsumerWarps;
-    }
+    if (warp < kConsumerWarps) { consumer_role(s, warp, V, status); return; }
+    const int helper = warp - kConsumerWarps;
     if (helper == kHelperIssuer) issuer_role(s, V, aligned, status);
     else if (helper == kHelperFetcher) fetcher_role(s, src, status);
     else if (helper == kHelperLayer) sink.layer_loop(s.layer);
+    else if (helper < kHelperFirstFinisher) sink.layer_assist(s.layer, helper - kHelperLayer);
     else finisher_role(s, sink, helper - kHelperFirstFinisher, V, k, aligned, status);
 }
 

@@ -22,6 +22,8 @@
 // are redone by the finisher warp with an exact radix-select path that re-reads the whole row.
 #pragma once
 
+#include <cstddef>
+
 #include "common.cuh"
 
 namespace ot {
@@ -61,14 +63,19 @@ struct alignas(16) RowSlot {
     int warpE[kConsumerWarps];
 };
 
-struct FinScratch {                // private to one finisher warp
+struct alignas(16) FinScratch {    // private to one finisher warp (hist is cleared and read with 16-byte accesses)
     unsigned long long cand[kCandCap];         // candidate keys of the row in hand, unordered
     int hist[256];
     int flist[kMaxFlag];                       // flagged thread ids
     int cand_count;
 };
 
-struct alignas(16) LayerScratch {  // private to the layer warp of a CTA
+struct LayerJob {                  // what the layer warp hands its assistants (kind 0: leave)
+    int kind, d, fsize, n, k, kk;
+    double* cand_phat; int32_t* cand_tok; int32_t* T_tok; int32_t* T_par; double* T_phat;
+};
+
+struct alignas(16) LayerScratch {  // private to the layer team of a CTA
     unsigned long long keys[1024 + 2];         // staged candidate keys, then the keys of R + layer
     unsigned long long lkeys[kMaxN];           // keys of the new layer, slot order
     double vals[kMaxN];                        // path values of the new running top-n
@@ -77,9 +84,14 @@ struct alignas(16) LayerScratch {  // private to the layer warp of a CTA
     int rsel[kMaxN];                           // gids of the new running top-n, ascending
     int ltok[kMaxN];                           // tokens of the new layer, slot order
     int hist[256];
+    int thist[3][256];                         // the team's digit counts, rotating (all zero between selections)
+    unsigned long long red_or[kTeamWarps], red_and[kTeamWarps];
+    int scan_a[kTeamWarps], scan_b[kTeamWarps];
+    LayerJob job;
 };
 
 static_assert(sizeof(RowSlot) % 16 == 0, "slots must keep 16-byte alignment in an array");
+static_assert(sizeof(FinScratch) % 16 == 0 && offsetof(FinScratch, hist) % 16 == 0, "hist must be 16-byte aligned in every finisher's scratch");
 // rows between "descriptor written" and "finisher has its copy": kDesc known + 1 streaming + kSlots handed on
 static_assert(kDescRing >= kDesc + 1 + kSlots + 1, "descriptor ring too short");
 
@@ -237,26 +249,29 @@ __device__ __forceinline__ unsigned long long warp_sort32_desc(unsigned long lon
     return v;
 }
 
-// k-th largest of the 16-bit keys key[0..kPerLane) held by every lane (32*kPerLane keys in all):
-// two 8-bit radix passes over a shared histogram.  1 <= k <= number of keys.
-__device__ __forceinline__ uint32_t warp_kth_largest16(const uint32_t (&key)[kPerLane], int k, int* hist) {
+// The finisher's code is walked once per row, by several warps at different places at once, next to
+// the consumers' loop: its size decides how often instructions have to be fetched again.  So its
+// common path is kept short (packed 16-bit operations, loops instead of unrolled sequences), and
+// everything rare sits in functions of its own that are not inlined.
+
+// k-th largest of a slot's per-thread keys (lane l owns tkey[16 l .. 16 l + 16)): two 8-bit radix
+// passes over a shared histogram.  1 <= k <= 512.  Rare: only when the maxima spread over more
+// than 256 key values.
+__device__ __noinline__ uint32_t warp_kth_largest16(const uint16_t* tkey, int k, int* hist) {
     const int lane = threadIdx.x & 31;
     uint32_t prefix = 0;
     int need = k;
-#pragma unroll
     for (int pass = 1; pass >= 0; --pass) {
-#pragma unroll
         for (int j = 0; j < 8; ++j) hist[lane * 8 + j] = 0;
         __syncwarp();
-#pragma unroll
-        for (int j = 0; j < kPerLane; ++j)
-            if (pass == 1 || (key[j] >> 8) == prefix) atomicAdd(&hist[(key[j] >> (8 * pass)) & 255u], 1);
+        for (int j = 0; j < kPerLane; ++j) {
+            const uint32_t key = tkey[lane * kPerLane + j];
+            if (pass == 1 || (key >> 8) == prefix) atomicAdd(&hist[(key >> (8 * pass)) & 255u], 1);
+        }
         __syncwarp();
         int c[8], mine = 0;
-#pragma unroll
         for (int j = 0; j < 8; ++j) { c[j] = hist[lane * 8 + j]; mine += c[j]; }
         int incl = mine;                                   // suffix sums over lanes from the top
-#pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
             if (lane + o < 32) incl += u;
@@ -265,14 +280,9 @@ __device__ __forceinline__ uint32_t warp_kth_largest16(const uint32_t (&key)[kPe
         const bool here = above < need && need <= incl;
         int bin = 0, nd = 0;
         if (here) {
-            int a = above;
-#pragma unroll
-            for (int b = 7; b >= 0; --b) {                 // highest bin whose suffix count reaches need
-                if (nd == 0) {
-                    if (a + c[b] >= need) { bin = lane * 8 + b; nd = need - a; }
-                    else a += c[b];
-                }
-            }
+            int a = above, bb = 7;
+            while (bb > 0 && a + c[bb] < need) { a += c[bb]; --bb; }
+            bin = lane * 8 + bb; nd = need - a;
         }
         const int src = __ffs(__ballot_sync(0xFFFFFFFFu, here)) - 1;
         bin = __shfl_sync(0xFFFFFFFFu, bin, src);
@@ -354,6 +364,11 @@ __device__ __noinline__ void row_exact_warp(FinScratch& f, const uint16_t* row, 
 
 // One 16-byte vector of the row (8 logits starting at token 8*vi) as four packed words; logits at or
 // beyond V read as -inf.  `aligned` rows take one vector load, others eight scalar loads.
+__device__ __noinline__ uint4 load_row_vec_scalar(const uint16_t* row, int vi, int V) {
+    uint32_t h[8];
+    for (int e = 0; e < 8; ++e) h[e] = (vi * 8 + e < V) ? (uint32_t)__ldg(row + vi * 8 + e) : 0xFF80u;
+    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+}
 __device__ __forceinline__ uint4 load_row_vec(const uint16_t* row, int vi, int V, bool aligned) {
     if (aligned) {
         uint4 v;
@@ -361,10 +376,29 @@ __device__ __forceinline__ uint4 load_row_vec(const uint16_t* row, int vi, int V
                      : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(reinterpret_cast<const uint4*>(row) + vi));
         return v;
     }
-    uint32_t h[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) h[e] = (vi * 8 + e < V) ? (uint32_t)__ldg(row + vi * 8 + e) : 0xFF80u;
-    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+    return load_row_vec_scalar(row, vi, V);
+}
+
+__device__ __noinline__ double exp_f64(double x) { return exp(x); }    // one copy of the routine for all its callers
+
+// bf16x2 "a >= b" per half: 0xFFFF where true
+__device__ __forceinline__ uint32_t ge_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("set.ge.u32.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// Ranks M <= 64 candidates (f.cand[0..M), distinct keys) and gives lane j < kk the j-th largest with
+// its probability.  S is the row's sum without the candidates unless `exact`.  The common case, up
+// to one candidate per lane, ranks by counting; more than 32 are sorted (rare).
+__device__ __noinline__ void finish_many(FinScratch& f, int M, int kk, double m, double S, bool exact, RowOut& out) {
+    const int lane = threadIdx.x & 31;
+    unsigned long long x0 = f.cand[lane], x1 = lane + 32 < M ? f.cand[lane + 32] : 0ull;
+    warp_sort64_desc(x0, x1);
+    const double e0 = exp_f64((double)cand_logit(x0) - m);
+    const double e1 = x1 ? exp_f64((double)cand_logit(x1) - m) : 0.0;
+    if (!exact) S += (double)warp_sum_u64(__double2ull_rn(e0 * kFixScale) + __double2ull_rn(e1 * kFixScale)) / kFixScale;
+    if (lane < kk) { out.tok = (int32_t)cand_token(x0); out.p = e0 / S; }
 }
 
 // Turns a finished slot into the row's k winners.  Whole finisher warp; f is its private scratch.
@@ -373,24 +407,19 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
     const int kk = k < V ? k : V;
     const int nvec = (V + 7) >> 3;
 
-    // this lane's 16 consecutive threads all belong to consumer warp lane / 2
-    uint32_t key[kPerLane];
+    // this lane's 16 consecutive threads all belong to consumer warp lane / 2; two 16-bit keys per word
+    uint32_t kw[kPerLane / 2];
     {
         const uint4* kp = reinterpret_cast<const uint4*>(&slot.tkey[lane * kPerLane]);
-#pragma unroll
-        for (int q = 0; q < kPerLane / 8; ++q) {
-            const uint4 w = kp[q];
-            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { key[q * 8 + 2 * i] = ww[i] & 0xFFFFu; key[q * 8 + 2 * i + 1] = ww[i] >> 16; }
-        }
+        const uint4 a = kp[0], b = kp[1];
+        kw[0] = a.x; kw[1] = a.y; kw[2] = a.z; kw[3] = a.w; kw[4] = b.x; kw[5] = b.y; kw[6] = b.z; kw[7] = b.w;
     }
     const int myE = slot.warpE[lane >> 1];
     const int emax = __reduce_max_sync(0xFFFFFFFFu, myE);
-    uint32_t mk = 0;
+    uint32_t mk = kw[0];
 #pragma unroll
-    for (int j = 0; j < kPerLane; ++j) mk = max(mk, key[j]);
-    mk = __reduce_max_sync(0xFFFFFFFFu, mk);
+    for (int q = 1; q < kPerLane / 2; ++q) mk = __vmaxu2(mk, kw[q]);
+    mk = __reduce_max_sync(0xFFFFFFFFu, max(mk & 0xFFFFu, mk >> 16));
 
     // tau: the kk-th largest per-thread maximum.  The maxima of a row lie close together, so a
     // histogram with one bin per key value over the 256 values below the largest usually holds kk
@@ -398,16 +427,19 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
     uint32_t tau_key;
     {
         const uint32_t base = mk > 255u ? mk - 255u : 0u;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) f.hist[lane * 8 + j] = 0;
+        uint4* hp = reinterpret_cast<uint4*>(&f.hist[lane * 8]);
+        hp[0] = make_uint4(0, 0, 0, 0); hp[1] = make_uint4(0, 0, 0, 0);
         __syncwarp();
 #pragma unroll
-        for (int j = 0; j < kPerLane; ++j)
-            if (key[j] >= base) atomicAdd(&f.hist[key[j] - base], 1);
+        for (int q = 0; q < kPerLane / 2; ++q) {
+            const uint32_t lo = kw[q] & 0xFFFFu, hi = kw[q] >> 16;
+            if (lo >= base) atomicAdd(&f.hist[lo - base], 1);
+            if (hi >= base) atomicAdd(&f.hist[hi - base], 1);
+        }
         __syncwarp();
-        int c[8], mine = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) { c[j] = f.hist[lane * 8 + j]; mine += c[j]; }
+        const uint4 c0 = hp[0], c1 = hp[1];
+        const int c[8] = {(int)c0.x, (int)c0.y, (int)c0.z, (int)c0.w, (int)c1.x, (int)c1.y, (int)c1.z, (int)c1.w};
+        const int mine = ((c[0] + c[1]) + (c[2] + c[3])) + ((c[4] + c[5]) + (c[6] + c[7]));
         int incl = mine;                                   // suffix sums over lanes from the top
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -430,21 +462,25 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
         const unsigned hm = __ballot_sync(0xFFFFFFFFu, here);
         __syncwarp();
         if (hm) tau_key = base + (uint32_t)__shfl_sync(0xFFFFFFFFu, bin, __ffs(hm) - 1);
-        else tau_key = warp_kth_largest16(key, kk, f.hist);
+        else tau_key = warp_kth_largest16(slot.tkey, kk, f.hist);
     }
     bool exact = tau_key <= kOrdNegInf || emax >= kExpLimit || emax <= -kExpLimit;
 
-    // the sum of all threads' partial sums; flagged threads listed in thread order
+    // the sum of all threads' partial sums; flagged threads (maximum >= tau) listed in thread order
     uint32_t fmask = 0;
     float part32 = 0.0f;
     {
+        const uint32_t tau2 = tau_key | (tau_key << 16);
+#pragma unroll
+        for (int q = 0; q < kPerLane / 2; ++q) {
+            const uint32_t g = __vcmpgeu2(kw[q], tau2);    // 0xFFFF per key >= tau
+            fmask |= ((g & 1u) | ((g >> 15) & 2u)) << (2 * q);
+        }
         const float4* sp = reinterpret_cast<const float4*>(&slot.tsum[lane * kPerLane]);
 #pragma unroll
         for (int q = 0; q < kPerLane / 4; ++q) {
             const float4 t4 = sp[q];
             part32 += (t4.x + t4.y) + (t4.z + t4.w);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) fmask |= key[q * 4 + i] >= tau_key ? (1u << (q * 4 + i)) : 0u;
         }
     }
     int nflag = 0;
@@ -468,41 +504,47 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
         // their tokens.  A candidate's term is already inside its thread's partial sum; the same
         // approximate term is taken out again here (the two differ by rounding of the exponent, a
         // few 1e-8 of the term), and the candidate comes back below with an exact exponential.
-        const float tau_f = bf16_bits_to_float(ord16_inv(tau_key));
+        // Work item i: flagged thread i mod P (P = nflag rounded up to a power of two), vector i / P.
+        const uint32_t tau_bits = ord16_inv(tau_key);
+        const float tau_f = bf16_bits_to_float(tau_bits);
+        const uint32_t tau_b2 = tau_bits | (tau_bits << 16);
         const int nchunks = (V + kChunkElems - 1) / kChunkElems;
         const int vpt = nchunks * kVecPerThread;
-        const int total = nflag * vpt;
+        const int lg = nflag > 1 ? 32 - __clz(nflag - 1) : 0;
+        const int total = vpt << lg;
         const float negE = -(float)emax;
         float sub = 0.0f;
+#pragma unroll 1
         for (int i0 = 0; i0 < total; i0 += 32 * 4) {
             uint4 w[4];
             int vis[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int idx = i0 + u * 32 + lane;
+                const int fi = idx & ((1 << lg) - 1), j = idx >> lg;
                 vis[u] = -1;
                 w[u] = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-                if (idx < total) {
-                    const int fi = idx / vpt, j = idx - fi * vpt;
+                if (idx < total && fi < nflag) {
                     const int vi = (j / kVecPerThread) * kChunkVecs + (j % kVecPerThread) * kConsumers + f.flist[fi];
                     if (vi < nvec) { vis[u] = vi; w[u] = load_row_vec(row, vi, V, aligned); }
                 }
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const uint32_t m2 = max_bf16x2(max_bf16x2(w[u].x, w[u].y), max_bf16x2(w[u].z, w[u].w));
-                const float vm = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
-                if (vis[u] < 0 || !(vm >= tau_f)) continue;                       // most vectors hold no candidate
-                const uint32_t ww[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const uint32_t bits = (e & 1) ? (ww[e >> 1] >> 16) : (ww[e >> 1] & 0xFFFFu);
-                    const float x = bf16_bits_to_float(bits);
-                    if (x >= tau_f) {
-                        const int pos = atomicAdd(&f.cand_count, 1);
-                        if (pos < kCandCap) f.cand[pos] = cand_key(bits, (uint32_t)(vis[u] * 8 + e));
-                        sub += ex2_approx(fmaf(x, kLog2e, negE));
-                    }
+                const uint32_t gx = ge_bf16x2(w[u].x, tau_b2), gy = ge_bf16x2(w[u].y, tau_b2);
+                const uint32_t gz = ge_bf16x2(w[u].z, tau_b2), gw = ge_bf16x2(w[u].w, tau_b2);
+                // bit e of m8: element e of the vector is a candidate (most vectors hold none)
+                uint32_t m8 = ((gx & 1u) | ((gx >> 15) & 2u)) | (((gy & 1u) | ((gy >> 15) & 2u)) << 2) |
+                              (((gz & 1u) | ((gz >> 15) & 2u)) << 4) | (((gw & 1u) | ((gw >> 15) & 2u)) << 6);
+                if (vis[u] < 0) m8 = 0;
+                while (m8) {
+                    const int e = __ffs(m8) - 1;
+                    m8 &= m8 - 1;
+                    const uint32_t word = e < 4 ? (e < 2 ? w[u].x : w[u].y) : (e < 6 ? w[u].z : w[u].w);
+                    const uint32_t bits = (e & 1) ? (word >> 16) : (word & 0xFFFFu);
+                    const int pos = atomicAdd(&f.cand_count, 1);
+                    if (pos < kCandCap) f.cand[pos] = cand_key(bits, (uint32_t)(vis[u] * 8 + e));
+                    sub += ex2_approx(fmaf(bf16_bits_to_float(bits), kLog2e, negE));
                 }
             }
         }
@@ -513,7 +555,7 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
             // Bulk terms are 2^(fl(x*L32) - E) with L32 the fp32 log2(e); wanted e^(x-m) = 2^((x-m)*L).
             // The exponent gap E - m*L + x*(L - L32) is evaluated at a typical bulk logit x = tau - 2.
             const double gap = (double)emax - m * kLog2eD + ((double)tau_f - 2.0) * (kLog2eD - (double)kLog2e);
-            S = warp_sum(part - (double)sub) * exp2(gap);
+            S = warp_sum(part - (double)sub) * exp_f64(gap * 0.693147180559945309417);
         }
     }
     if (exact) {
@@ -524,18 +566,24 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
 
     out.kk = kk; out.tok = -1; out.p = 0.0;
     if (M <= 32) {
-        // one candidate per lane: sort, then every lane's exponential once
-        const unsigned long long mine = warp_sort32_desc(lane < M ? f.cand[lane] : 0ull);
-        const double e = lane < M ? exp((double)cand_logit(mine) - m) : 0.0;
+        // one candidate per lane: every lane's exponential once; its rank is the number of larger
+        // candidates (keys are distinct), and rank j's token and term go to lane j through the scratch
+        const unsigned long long mine = lane < M ? f.cand[lane] : 0ull;
+        const double e = lane < M ? exp_f64((double)cand_logit(mine) - m) : 0.0;
         if (!exact) S += (double)warp_sum_u64(__double2ull_rn(e * kFixScale)) / kFixScale;   // integer sum: order free
-        if (lane < kk) { out.tok = (int32_t)cand_token(mine); out.p = e / S; }
+        int rank = 0;
+#pragma unroll 1
+        for (int j = 0; j < M; ++j) rank += __shfl_sync(0xFFFFFFFFu, mine, j) > mine ? 1 : 0;
+        __syncwarp();
+        if (lane < M) { f.cand[rank] = mine; f.cand[32 + rank] = (unsigned long long)__double_as_longlong(e); }
+        __syncwarp();
+        if (lane < kk) {
+            out.tok = (int32_t)cand_token(f.cand[lane]);
+            out.p = __longlong_as_double((long long)f.cand[32 + lane]) / S;
+        }
+        __syncwarp();
     } else {
-        unsigned long long x0 = f.cand[lane], x1 = lane + 32 < M ? f.cand[lane + 32] : 0ull;
-        warp_sort64_desc(x0, x1);
-        const double e0 = exp((double)cand_logit(x0) - m);
-        const double e1 = x1 ? exp((double)cand_logit(x1) - m) : 0.0;
-        S += (double)warp_sum_u64(__double2ull_rn(e0 * kFixScale) + __double2ull_rn(e1 * kFixScale)) / kFixScale;
-        if (lane < kk) { out.tok = (int32_t)cand_token(x0); out.p = e0 / S; }
+        finish_many(f, M, kk, m, S, exact, out);
     }
 }
 

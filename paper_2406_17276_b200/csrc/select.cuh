@@ -265,6 +265,160 @@ __device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int f
     return nl;
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same layer selection by the layer team (kTeam threads: the layer warp and its assistants;
+// thread tt of the team).  Every step that loops over the candidates is split over the team;
+// the decisions in between are computed by each warp for itself from the same shared-memory
+// counts, so all warps take the same path and meet at the same barriers.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ int team_excl_scan(int v, int* wtot, int tw, int& total) {
+    int wt;
+    const int base = warp_excl_scan(v, wt);
+    if ((threadIdx.x & 31) == 0) wtot[tw] = wt;
+    team_sync();
+    int before = 0;
+    total = 0;
+#pragma unroll
+    for (int q = 0; q < kTeamWarps; ++q) { const int x = wtot[q]; total += x; before += q < tw ? x : 0; }
+    return base + before;
+}
+
+// Threshold of the `need` largest keys among s.keys[0..N) (0 = not an element); see
+// warp_radix_select for the result and the shortcuts.  The digit counts rotate through three
+// arrays that are all zero on entry: pass p counts into array p % 3 and clears the one pass p-1
+// read, so one barrier per pass is enough.  Returns the array that is left non-zero (the caller
+// clears it after its next barrier), or -1.
+__device__ int team_radix_select(LayerScratch& s, int N, int need, int tt, unsigned long long key_or, unsigned long long key_and,
+                                 unsigned long long& thr, int& need_eq) {
+    const int lane = threadIdx.x & 31;
+    const unsigned long long diff = key_or ^ key_and;
+    if (diff == 0ull) { thr = key_or; need_eq = need; return -1; }       // all elements equal
+    int top = 64 - __clzll((long long)diff);                             // the low `top` bits vary
+    unsigned long long prefix = top == 64 ? 0ull : ((key_or >> top) << top);
+    int pass = 0;
+    while (top > 0) {
+        const int wbits = top < 8 ? top : 8, shift = top - wbits;
+        const unsigned int dmask = (1u << wbits) - 1u;
+        int* hist = s.thist[pass % 3];
+        for (int i = tt; i < N; i += kTeam) {
+            const unsigned long long key = s.keys[i];
+            const bool match = key != 0ull && (top == 64 || (key >> top) == (prefix >> top));
+            if (match) atomicAdd(&hist[(int)((unsigned int)(key >> shift) & dmask)], 1);
+        }
+        team_sync();
+        int c[8], mine = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = hist[lane * 8 + j]; mine += c[j]; }
+        {   // the array read one pass ago is free again
+            int* z = s.thist[(pass + 2) % 3];
+            z[tt] = 0; z[tt + kTeam] = 0;
+        }
+        int incl = mine;                                   // suffix sums over lanes from the top
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
+            if (lane + o < 32) incl += u;
+        }
+        const int above = incl - mine;
+        const bool here = above < need && need <= incl;
+        int bin = 0, nd = 0, cb = 0;
+        if (here) {
+            int a = above;
+            bin = lane * 8;
+#pragma unroll
+            for (int b = 7; b >= 0; --b) {                 // highest bin whose suffix count reaches need
+                if (nd == 0) {
+                    if (a + c[b] >= need) { bin = lane * 8 + b; nd = need - a; cb = c[b]; }
+                    else a += c[b];
+                }
+            }
+        }
+        const int src = __ffs(__ballot_sync(0xFFFFFFFFu, here)) - 1;
+        bin = __shfl_sync(0xFFFFFFFFu, bin, src);
+        need = __shfl_sync(0xFFFFFFFFu, nd, src);
+        cb = __shfl_sync(0xFFFFFFFFu, cb, src);
+        prefix |= (unsigned long long)bin << shift;
+        top = shift;
+        ++pass;
+        if (cb == need && prefix != 0ull) { thr = prefix - 1ull; need_eq = 0; return (pass - 1) % 3; }   // the whole bin belongs
+    }
+    thr = prefix;
+    need_eq = need;
+    return (pass - 1) % 3;
+}
+
+// The team's part of a layer selection (N = fsize * k <= 1024; the candidates were staged into s
+// by the layer warp).  On return (after a last barrier) the new layer's nodes are in T and its
+// tokens and keys in s.ltok / s.lkeys.  Returns nl.
+__device__ int select_layer_team(LayerScratch& s, const LayerJob& j, int tt, int* status) {
+    const int lane = threadIdx.x & 31, tw = tt >> 5;
+    const int N = j.fsize * j.k;
+    const int nvalid = j.fsize * j.kk;
+    const int nl = nvalid < j.n ? nvalid : j.n;
+    const int gid0 = (j.d - 1) * j.n;
+    const unsigned long long* gph = reinterpret_cast<const unsigned long long*>(j.cand_phat);
+    const unsigned int* gtk = reinterpret_cast<const unsigned int*>(j.cand_tok);
+    unsigned long long ko = 0ull, ka = ~0ull;
+    for (int i = tt; i < N; i += kTeam) {
+        // words that were not there yet when they were staged are read again until they are (bounded)
+        unsigned long long x = s.keys[i];
+        for (int t = 0; !(x >> 63) && t < (1 << 22); ++t) x = ld_relaxed_u64(&gph[i]);
+        if (!(x >> 63)) { set_status(status, kErrTimeout); x = ~0ull; }
+        const unsigned long long key = x == ~0ull ? 0ull : (x & 0x7FFFFFFFFFFFFFFFull) + 1ull;
+        s.keys[i] = key;
+        if (key) { ko |= key; ka &= key; }
+        unsigned int t32 = (unsigned int)s.toks[i];
+        for (int t = 0; !(t32 >> 31) && t < (1 << 22); ++t) t32 = ld_relaxed_u32(&gtk[i]);
+        if (!(t32 >> 31)) { set_status(status, kErrTimeout); t32 = ~0u; }
+        s.toks[i] = (int)t32;
+    }
+    ko = warp_or_u64(ko); ka = warp_and_u64(ka);
+    if (lane == 0) { s.red_or[tw] = ko; s.red_and[tw] = ka; }
+    team_sync();
+    ko = 0ull; ka = ~0ull;
+#pragma unroll
+    for (int q = 0; q < kTeamWarps; ++q) { ko |= s.red_or[q]; ka &= s.red_and[q]; }
+    // every candidate has been read: the arrays are free for the next layer's rows once they are zero again
+    for (int i = tt * 2; i < N; i += 2 * kTeam) *reinterpret_cast<uint4*>(&j.cand_phat[i]) = make_uint4(0, 0, 0, 0);
+    for (int i = tt * 4; i < N; i += 4 * kTeam) *reinterpret_cast<uint4*>(&j.cand_tok[i]) = make_uint4(0, 0, 0, 0);
+    unsigned long long thr;
+    int need_eq;
+    const int dirty = team_radix_select(s, N, nl, tt, ko, ka, thr, need_eq);
+    // ordered compaction: thread tt owns a contiguous stretch of candidates
+    const int per = (N + kTeam - 1) / kTeam;
+    const int lo = min(tt * per, N), hi = min(lo + per, N);
+    int gt = 0, eq = 0;
+    for (int i = lo; i < hi; ++i) {
+        const unsigned long long key = s.keys[i];
+        gt += key > thr ? 1 : 0;
+        eq += key == thr ? 1 : 0;
+    }
+    int total_eq, total;
+    const int eq_before = team_excl_scan(eq, s.scan_a, tw, total_eq);
+    if (dirty >= 0) { s.thist[dirty][tt] = 0; s.thist[dirty][tt + kTeam] = 0; }     // everyone is past the last pass
+    int eq_take = need_eq - eq_before;
+    eq_take = eq_take < 0 ? 0 : (eq_take > eq ? eq : eq_take);
+    int pos = team_excl_scan(gt + eq_take, s.scan_b, tw, total);
+    for (int i = lo; i < hi; ++i) {
+        const unsigned long long key = s.keys[i];
+        bool take = key > thr;
+        if (key == thr && eq_take > 0) { take = true; --eq_take; }
+        if (take) {
+            const unsigned int t32 = (unsigned int)s.toks[i];
+            const int tok = t32 == ~0u ? -1 : (int)(t32 & 0x7FFFFFFFu);
+            j.T_tok[gid0 + pos] = tok;
+            s.ltok[pos] = tok;
+            j.T_par[gid0 + pos] = i / j.k;
+            j.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
+            s.lkeys[pos] = key;
+            ++pos;
+        }
+    }
+    if (total != nl) set_status(status, kErrInternal);
+    team_sync();
+    return nl;
+}
+
 // Layer job, second half: the running top-n and E_sub(T, n) with the new layer (left in s by
 // select_layer_warp), the loop test of Algorithm 1, and the packed tree if the sequence is
 // finished.  All layers of a sequence are handled by the same warp, in order.  Returns true if the
