@@ -291,7 +291,7 @@ struct BuildSink {
             long long t0 = clock64();
             while (live > 0) {
                 bool progressed = false;
-#pragma unroll
+#pragma unroll 1                                          // one copy of the body: it is long, and instruction fetch is what the helper warps wait for
                 for (int q = 0; q < kOwn; ++q) {
                     if (cur_d[q] == 0) continue;
                     const int b = b0 + q * (int)gridDim.x;

@@ -179,7 +179,7 @@ __device__ __forceinline__ void stage_layer_candidates(LayerScratch& s, const Se
 // Layer job, first half.  After all rows of layer d (1-based) of one sequence are expanded: the
 // next layer = the nl candidates of largest path value, stored in candidate-index order (nodes
 // gid0 .. gid0+nl of T; tokens and keys also left in s.ltok / s.lkeys).  Whole layer warp; s is its scratch; fsize = rows of the layer.  Returns nl.
-__device__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int fsize, int n, int k, int kk, int* status) {
+__device__ __noinline__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int fsize, int n, int k, int kk, int* status) {
     const int lane = threadIdx.x & 31;
     int* hist = s.hist;
     const int N = fsize * k;
@@ -350,7 +350,7 @@ __device__ int team_radix_select(LayerScratch& s, int N, int need, int tt, unsig
 // The team's part of a layer selection (N = fsize * k <= 1024; the candidates were staged into s
 // by the layer warp).  On return (after a last barrier) the new layer's nodes are in T and its
 // tokens and keys in s.ltok / s.lkeys.  Returns nl.
-__device__ int select_layer_team(LayerScratch& s, const LayerJob& j, int tt, int* status) {
+__device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j, int tt, int* status) {
     const int lane = threadIdx.x & 31, tw = tt >> 5;
     const int N = j.fsize * j.k;
     const int nvalid = j.fsize * j.kk;
@@ -423,7 +423,7 @@ __device__ int select_layer_team(LayerScratch& s, const LayerJob& j, int tt, int
 // select_layer_warp), the loop test of Algorithm 1, and the packed tree if the sequence is
 // finished.  All layers of a sequence are handled by the same warp, in order.  Returns true if the
 // sequence continues with layer d+1, false if it is finished (outputs written).
-__device__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
+__device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
                                     int max_depth, float delta, int* status) {
     const int lane = threadIdx.x & 31;
     int* hist = s.hist;
