@@ -98,6 +98,14 @@ __device__ void fetcher_role(CtaSmem& s, Source& src, int* status) {
 }
 
 // ---- issuer warp -------------------------------------------------------------------------------
+// A chunk of a row that bulk copies cannot take (see issuer_role), by the whole warp; rare, out of line.
+__device__ __noinline__ void copy_chunk_plain(uint16_t* stage, const uint16_t* src, int ne) {
+    const int lane = threadIdx.x & 31;
+    const int padded = (ne + 7) & ~7;
+    for (int i = lane; i < padded; i += 32) stage[i] = i < ne ? __ldg(src + i) : (uint16_t)0xFF80u;
+    __syncwarp();
+}
+
 // With `aligned` false (table base or row pitch not 16-byte aligned) the whole warp copies the
 // chunk with ordinary loads instead of a bulk copy.
 __device__ void issuer_role(CtaSmem& s, int V, bool aligned, int* status) {
@@ -124,10 +132,7 @@ __device__ void issuer_role(CtaSmem& s, int V, bool aligned, int* status) {
                     bulk_load(&s.stage[st][0], row + (size_t)c * kChunkElems, (uint32_t)ne * 2u, &s.full_bar[st]);
                 }
             } else {
-                const int padded = (ne + 7) & ~7;
-                for (int i = lane; i < padded; i += 32)
-                    s.stage[st][i] = i < ne ? __ldg(row + (size_t)c * kChunkElems + i) : (uint16_t)0xFF80u;
-                __syncwarp();
+                copy_chunk_plain(&s.stage[st][0], row + (size_t)c * kChunkElems, ne);
                 if (lane == 0) mbar_arrive(&s.full_bar[st]);
             }
         }

@@ -43,6 +43,7 @@ __device__ void warp_radix_select(KeyFn keyf, int N, int need, int* hist, unsign
 #pragma unroll
         for (int j = 0; j < 8; ++j) hist[lane * 8 + j] = 0;
         __syncwarp();
+        #pragma unroll 1
         for (int i = lane; i < N; i += 32) {
             const unsigned long long key = keyf(i);
             const bool match = key != 0ull && (top == 64 || (key >> top) == (prefix >> top));
@@ -92,6 +93,7 @@ __device__ int warp_compact_selected(KeyFn keyf, int N, unsigned long long thr, 
     const int lane = threadIdx.x & 31;
     const unsigned below = (1u << lane) - 1u;
     int eq_seen = 0, taken = 0;
+    #pragma unroll 1
     for (int i0 = 0; i0 < N; i0 += 32) {
         const int i = i0 + lane;
         const unsigned long long key = i < N ? keyf(i) : 0ull;
@@ -129,6 +131,7 @@ __device__ int warp_compact_selected_blocked(KeyFn keyf, int N, unsigned long lo
     eq_take = eq_take < 0 ? 0 : (eq_take > eq ? eq : eq_take);
     int pos = warp_excl_scan(gt + eq_take, total);
     if (gt + eq_take > 0) {
+        #pragma unroll 1
         for (int i = lo; i < hi; ++i) {
             const unsigned long long key = keyf(i);
             bool take = key > thr;
@@ -137,6 +140,7 @@ __device__ int warp_compact_selected_blocked(KeyFn keyf, int N, unsigned long lo
         }
     }
     __syncwarp();
+    #pragma unroll 1
     for (int q = lane; q < total; q += 32) emit(q, idx[q]);
     __syncwarp();
     return total;
@@ -172,7 +176,9 @@ __device__ __forceinline__ void stage_layer_candidates(LayerScratch& s, const Se
     if (N > 1024) return;
     const unsigned long long* gph = reinterpret_cast<const unsigned long long*>(w.cand_phat);
     const unsigned int* gtk = reinterpret_cast<const unsigned int*>(w.cand_tok);
+    #pragma unroll 1
     for (int i = lane * 2; i < N; i += 64) cp_async_16(&s.keys[i], &gph[i]);
+    #pragma unroll 1
     for (int i = lane * 4; i < N; i += 128) cp_async_16(&s.toks[i], &gtk[i]);
 }
 
@@ -228,7 +234,9 @@ __device__ __noinline__ int select_layer_warp(LayerScratch& s, const SeqWork& w,
         }
         __syncwarp();
         // the arrays are free for the next layer's rows once they are zero again
+        #pragma unroll 1
         for (int i = lane * 2; i < N; i += 64) *reinterpret_cast<uint4*>(&w.cand_phat[i]) = make_uint4(0, 0, 0, 0);
+        #pragma unroll 1
         for (int i = lane * 4; i < N; i += 128) *reinterpret_cast<uint4*>(&w.cand_tok[i]) = make_uint4(0, 0, 0, 0);
         auto skey = [&](int i) -> unsigned long long { return s.keys[i]; };
         warp_radix_select(skey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
@@ -243,6 +251,7 @@ __device__ __noinline__ int select_layer_warp(LayerScratch& s, const SeqWork& w,
         });
     } else {
         auto gkey = [&](int i) -> unsigned long long { return key_of(wait_phat(i)); };
+        #pragma unroll 1
         for (int i = lane; i < N; i += 32) {
             const unsigned long long key = gkey(i);
             if (key) { ko |= key; ka &= key; }
@@ -258,11 +267,28 @@ __device__ __noinline__ int select_layer_warp(LayerScratch& s, const SeqWork& w,
             s.lkeys[pos] = key;
         });
         __syncwarp();
+        #pragma unroll 1
         for (int i = lane * 2; i < N; i += 64) *reinterpret_cast<uint4*>(&w.cand_phat[i]) = make_uint4(0, 0, 0, 0);
+        #pragma unroll 1
         for (int i = lane * 4; i < N; i += 128) *reinterpret_cast<uint4*>(&w.cand_tok[i]) = make_uint4(0, 0, 0, 0);
     }
     __syncwarp();
     return nl;
+}
+
+// A candidate word that was not there yet when it was looked at is read again until it is (bounded).
+// Rare, so out of line.
+__device__ __noinline__ unsigned long long poll_phat_word(const unsigned long long* p, int* status) {
+    unsigned long long x = ld_relaxed_u64(p);
+    for (int t = 0; !(x >> 63) && t < (1 << 22); ++t) x = ld_relaxed_u64(p);
+    if (!(x >> 63)) { set_status(status, kErrTimeout); x = ~0ull; }
+    return x;
+}
+__device__ __noinline__ unsigned int poll_tok_word(const unsigned int* p, int* status) {
+    unsigned int x = ld_relaxed_u32(p);
+    for (int t = 0; !(x >> 31) && t < (1 << 22); ++t) x = ld_relaxed_u32(p);
+    if (!(x >> 31)) { set_status(status, kErrTimeout); x = ~0u; }
+    return x;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -300,6 +326,7 @@ __device__ int team_radix_select(LayerScratch& s, int N, int need, int tt, unsig
         const int wbits = top < 8 ? top : 8, shift = top - wbits;
         const unsigned int dmask = (1u << wbits) - 1u;
         int* hist = s.thist[pass % 3];
+        #pragma unroll 1
         for (int i = tt; i < N; i += kTeam) {
             const unsigned long long key = s.keys[i];
             const bool match = key != 0ull && (top == 64 || (key >> top) == (prefix >> top));
@@ -359,18 +386,16 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
     const unsigned long long* gph = reinterpret_cast<const unsigned long long*>(j.cand_phat);
     const unsigned int* gtk = reinterpret_cast<const unsigned int*>(j.cand_tok);
     unsigned long long ko = 0ull, ka = ~0ull;
+    #pragma unroll 1
     for (int i = tt; i < N; i += kTeam) {
         // words that were not there yet when they were staged are read again until they are (bounded)
         unsigned long long x = s.keys[i];
-        for (int t = 0; !(x >> 63) && t < (1 << 22); ++t) x = ld_relaxed_u64(&gph[i]);
-        if (!(x >> 63)) { set_status(status, kErrTimeout); x = ~0ull; }
+        if (!(x >> 63)) x = poll_phat_word(&gph[i], status);
         const unsigned long long key = x == ~0ull ? 0ull : (x & 0x7FFFFFFFFFFFFFFFull) + 1ull;
         s.keys[i] = key;
         if (key) { ko |= key; ka &= key; }
         unsigned int t32 = (unsigned int)s.toks[i];
-        for (int t = 0; !(t32 >> 31) && t < (1 << 22); ++t) t32 = ld_relaxed_u32(&gtk[i]);
-        if (!(t32 >> 31)) { set_status(status, kErrTimeout); t32 = ~0u; }
-        s.toks[i] = (int)t32;
+        if (!(t32 >> 31)) { t32 = poll_tok_word(&gtk[i], status); s.toks[i] = (int)t32; }
     }
     ko = warp_or_u64(ko); ka = warp_and_u64(ka);
     if (lane == 0) { s.red_or[tw] = ko; s.red_and[tw] = ka; }
@@ -379,7 +404,9 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
 #pragma unroll
     for (int q = 0; q < kTeamWarps; ++q) { ko |= s.red_or[q]; ka &= s.red_and[q]; }
     // every candidate has been read: the arrays are free for the next layer's rows once they are zero again
+    #pragma unroll 1
     for (int i = tt * 2; i < N; i += 2 * kTeam) *reinterpret_cast<uint4*>(&j.cand_phat[i]) = make_uint4(0, 0, 0, 0);
+    #pragma unroll 1
     for (int i = tt * 4; i < N; i += 4 * kTeam) *reinterpret_cast<uint4*>(&j.cand_tok[i]) = make_uint4(0, 0, 0, 0);
     unsigned long long thr;
     int need_eq;
@@ -388,6 +415,7 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
     const int per = (N + kTeam - 1) / kTeam;
     const int lo = min(tt * per, N), hi = min(lo + per, N);
     int gt = 0, eq = 0;
+    #pragma unroll 1
     for (int i = lo; i < hi; ++i) {
         const unsigned long long key = s.keys[i];
         gt += key > thr ? 1 : 0;
@@ -399,6 +427,7 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
     int eq_take = need_eq - eq_before;
     eq_take = eq_take < 0 ? 0 : (eq_take > eq ? eq : eq_take);
     int pos = team_excl_scan(gt + eq_take, s.scan_b, tw, total);
+    #pragma unroll 1
     for (int i = lo; i < hi; ++i) {
         const unsigned long long key = s.keys[i];
         bool take = key > thr;
@@ -419,59 +448,13 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
     return nl;
 }
 
-// Layer job, second half: the running top-n and E_sub(T, n) with the new layer (left in s by
-// select_layer_warp), the loop test of Algorithm 1, and the packed tree if the sequence is
-// finished.  All layers of a sequence are handled by the same warp, in order.  Returns true if the
-// sequence continues with layer d+1, false if it is finished (outputs written).
-__device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
-                                    int max_depth, float delta, int* status) {
+// Once per sequence, when it is finished: T_opt = the running top-n (s.rsel / s.vals, already in
+// (depth, parent's index, sibling rank) order), packed with parent indices.
+__device__ __noinline__ void pack_tree_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nR, int n, int max_depth,
+                                            double esub, int* status) {
     const int lane = threadIdx.x & 31;
-    int* hist = s.hist;
-    const int gid0 = (d - 1) * n;
-    unsigned long long thr;
-    int need_eq;
-    const int nR_old = d == 1 ? 0 : __ldcg(&w.st[kStNR]);
-    const double eprev = d == 1 ? 0.0 : __ldcg(w.E_prev);
-
-    // --- E_sub(T, n): the n largest path values among the previous top-n and the new layer ---
-    const int32_t* Rold = w.R + ((d - 1) & 1) * n;
-    int32_t* Rnew = w.R + (d & 1) * n;
-    const int NR = nR_old + nl;                           // <= 2n <= 512
-    const int nR = NR < n ? NR : n;
-    unsigned long long ko = 0ull, ka = ~0ull;
-#pragma unroll 4
-    for (int i = lane; i < NR; i += 32) {
-        int gid;
-        unsigned long long key;
-        if (i < nR_old) { gid = __ldcg(&Rold[i]); key = phat_key(__ldcg(&w.T_phat[gid])); }
-        else { gid = gid0 + (i - nR_old); key = s.lkeys[i - nR_old]; }
-        s.gids[i] = gid;
-        s.keys[i] = key;
-        ko |= key; ka &= key;
-    }
-    __syncwarp();
-    auto rkey = [&](int i) -> unsigned long long { return s.keys[i]; };
-    warp_radix_select(rkey, NR, nR, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
-    warp_compact_selected(rkey, NR, thr, need_eq, [&](int pos, int i) {
-        Rnew[pos] = s.gids[i];
-        s.rsel[pos] = s.gids[i];
-        s.vals[pos] = __longlong_as_double((long long)(s.keys[i] - 1ull));
-    });
-    __syncwarp();
-    double part = 0.0;
-    for (int i = lane; i < nR; i += 32) part += s.vals[i];
-    const double esub = warp_sum(part);                   // fixed order: lanes stride the packed order
-    const bool more = d < Dcap && (esub - eprev > (double)delta);     // loop test of Algorithm 1
-    if (out.esub_trace && lane == 0) out.esub_trace[d - 1] = esub;
-    if (lane == 0) {
-        w.st[kStNR] = nR;
-        *w.E_prev = esub;
-    }
-    __syncwarp();
-    if (more) return true;
-
-    // --- pack: T_opt = the running top-n, already in (depth, parent's index, sibling rank) order ---
     if (out.esub_trace) for (int i = d + lane; i < max_depth; i += 32) out.esub_trace[i] = 0.0;
+    #pragma unroll 1
     for (int i = lane; i < n; i += 32) {
         int32_t tok = -1, par = -1, dep = 0;
         double ph = 0.0;
@@ -494,6 +477,60 @@ __device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork&
         out.token[i] = tok; out.parent[i] = par; out.depth[i] = dep; out.phat[i] = ph;
     }
     if (lane == 0) { *out.n_sel = nR; *out.depth_reached = d; *out.expected_len = esub; }
+}
+
+// Layer job, second half: the running top-n and E_sub(T, n) with the new layer (left in s by
+// select_layer_warp), the loop test of Algorithm 1, and the packed tree if the sequence is
+// finished.  All layers of a sequence are handled by the same warp, in order.  Returns true if the
+// sequence continues with layer d+1, false if it is finished (outputs written).
+__device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
+                                    int max_depth, float delta, int* status) {
+    const int lane = threadIdx.x & 31;
+    int* hist = s.hist;
+    const int gid0 = (d - 1) * n;
+    unsigned long long thr;
+    int need_eq;
+    const int nR_old = d == 1 ? 0 : __ldcg(&w.st[kStNR]);
+    const double eprev = d == 1 ? 0.0 : __ldcg(w.E_prev);
+
+    // --- E_sub(T, n): the n largest path values among the previous top-n and the new layer ---
+    const int32_t* Rold = w.R + ((d - 1) & 1) * n;
+    int32_t* Rnew = w.R + (d & 1) * n;
+    const int NR = nR_old + nl;                           // <= 2n <= 512
+    const int nR = NR < n ? NR : n;
+    unsigned long long ko = 0ull, ka = ~0ull;
+    #pragma unroll 1
+    for (int i = lane; i < NR; i += 32) {
+        int gid;
+        unsigned long long key;
+        if (i < nR_old) { gid = __ldcg(&Rold[i]); key = phat_key(__ldcg(&w.T_phat[gid])); }
+        else { gid = gid0 + (i - nR_old); key = s.lkeys[i - nR_old]; }
+        s.gids[i] = gid;
+        s.keys[i] = key;
+        ko |= key; ka &= key;
+    }
+    __syncwarp();
+    auto rkey = [&](int i) -> unsigned long long { return s.keys[i]; };
+    warp_radix_select(rkey, NR, nR, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
+    warp_compact_selected(rkey, NR, thr, need_eq, [&](int pos, int i) {
+        Rnew[pos] = s.gids[i];
+        s.rsel[pos] = s.gids[i];
+        s.vals[pos] = __longlong_as_double((long long)(s.keys[i] - 1ull));
+    });
+    __syncwarp();
+    double part = 0.0;
+    #pragma unroll 1
+    for (int i = lane; i < nR; i += 32) part += s.vals[i];
+    const double esub = warp_sum(part);                   // fixed order: lanes stride the packed order
+    const bool more = d < Dcap && (esub - eprev > (double)delta);     // loop test of Algorithm 1
+    if (out.esub_trace && lane == 0) out.esub_trace[d - 1] = esub;
+    if (lane == 0) {
+        w.st[kStNR] = nR;
+        *w.E_prev = esub;
+    }
+    __syncwarp();
+    if (more) return true;
+    pack_tree_warp(s, w, out, d, nR, n, max_depth, esub, status);
     return false;
 }
 
