@@ -430,11 +430,10 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
         uint4* hp = reinterpret_cast<uint4*>(&f.hist[lane * 8]);
         hp[0] = make_uint4(0, 0, 0, 0); hp[1] = make_uint4(0, 0, 0, 0);
         __syncwarp();
-#pragma unroll
-        for (int q = 0; q < kPerLane / 2; ++q) {
-            const uint32_t lo = kw[q] & 0xFFFFu, hi = kw[q] >> 16;
-            if (lo >= base) atomicAdd(&f.hist[lo - base], 1);
-            if (hi >= base) atomicAdd(&f.hist[hi - base], 1);
+#pragma unroll 1
+        for (int q = 0; q < kPerLane; ++q) {               // (keys from the slot again: a loop, not sixteen copies)
+            const uint32_t key = slot.tkey[lane * kPerLane + q];
+            if (key >= base) atomicAdd(&f.hist[key - base], 1);
         }
         __syncwarp();
         const uint4 c0 = hp[0], c1 = hp[1];
@@ -529,23 +528,28 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
                     if (vi < nvec) { vis[u] = vi; w[u] = load_row_vec(row, vi, V, aligned); }
                 }
             }
+            // bit 8u+e of m32: element e of vector u is a candidate (most vectors hold none)
+            uint32_t m32 = 0;
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const uint32_t gx = ge_bf16x2(w[u].x, tau_b2), gy = ge_bf16x2(w[u].y, tau_b2);
                 const uint32_t gz = ge_bf16x2(w[u].z, tau_b2), gw = ge_bf16x2(w[u].w, tau_b2);
-                // bit e of m8: element e of the vector is a candidate (most vectors hold none)
-                uint32_t m8 = ((gx & 1u) | ((gx >> 15) & 2u)) | (((gy & 1u) | ((gy >> 15) & 2u)) << 2) |
-                              (((gz & 1u) | ((gz >> 15) & 2u)) << 4) | (((gw & 1u) | ((gw >> 15) & 2u)) << 6);
-                if (vis[u] < 0) m8 = 0;
-                while (m8) {
-                    const int e = __ffs(m8) - 1;
-                    m8 &= m8 - 1;
-                    const uint32_t word = e < 4 ? (e < 2 ? w[u].x : w[u].y) : (e < 6 ? w[u].z : w[u].w);
-                    const uint32_t bits = (e & 1) ? (word >> 16) : (word & 0xFFFFu);
-                    const int pos = atomicAdd(&f.cand_count, 1);
-                    if (pos < kCandCap) f.cand[pos] = cand_key(bits, (uint32_t)(vis[u] * 8 + e));
-                    sub += ex2_approx(fmaf(bf16_bits_to_float(bits), kLog2e, negE));
-                }
+                const uint32_t m8 = ((gx & 1u) | ((gx >> 15) & 2u)) | (((gy & 1u) | ((gy >> 15) & 2u)) << 2) |
+                                    (((gz & 1u) | ((gz >> 15) & 2u)) << 4) | (((gw & 1u) | ((gw >> 15) & 2u)) << 6);
+                m32 |= (vis[u] < 0 ? 0u : m8) << (8 * u);
+            }
+#pragma unroll 1
+            while (m32) {
+                const int e = __ffs(m32) - 1;
+                m32 &= m32 - 1;
+                const int u = e >> 3, h = e & 7;
+                const uint4 wu = u < 2 ? (u == 0 ? w[0] : w[1]) : (u == 2 ? w[2] : w[3]);
+                const int vi = u < 2 ? (u == 0 ? vis[0] : vis[1]) : (u == 2 ? vis[2] : vis[3]);
+                const uint32_t word = h < 4 ? (h < 2 ? wu.x : wu.y) : (h < 6 ? wu.z : wu.w);
+                const uint32_t bits = (h & 1) ? (word >> 16) : (word & 0xFFFFu);
+                const int pos = atomicAdd(&f.cand_count, 1);
+                if (pos < kCandCap) f.cand[pos] = cand_key(bits, (uint32_t)(vi * 8 + h));
+                sub += ex2_approx(fmaf(bf16_bits_to_float(bits), kLog2e, negE));
             }
         }
         __syncwarp();
