@@ -12,12 +12,12 @@
 // Nothing in that pass depends on a threshold, so consecutive rows stream without a bubble.
 //
 // A finisher warp then turns the 512 per-thread (max, sum) pairs into the row's result:
-//   * tau = k-th largest per-thread maximum: a lower bound of the row's k-th largest logit, so
-//     every winner lives in a thread whose maximum is >= tau ("flagged", about k of 512);
-//   * the flagged threads' vectors are read again (they are still in L2): logits >= tau become
-//     candidates, the others are summed like the bulk;
+//   * tau = a lower bound of the row's k-th largest logit, taken from the per-thread maxima, so
+//     every winner lives in a thread whose maximum is >= tau ("flagged", a few more than k of 512);
+//   * the flagged threads' vectors are read again (they are still in L2) to find the logits >= tau,
+//     the candidates, with their tokens; their approximate terms are taken out of the sums again;
 //   * candidates are ranked exactly on (bf16 bits, token id) and their exponentials taken in fp64;
-//     the unflagged threads' sums are combined in fp64; probabilities of the k winners follow.
+//     the threads' sums are combined in fp64; probabilities of the k winners follow.
 // Rows this cannot handle (fewer than k finite per-thread maxima, heavy ties, extreme magnitudes)
 // are redone by the finisher warp with an exact radix-select path that re-reads the whole row.
 #pragma once
@@ -254,45 +254,6 @@ __device__ __forceinline__ unsigned long long warp_sort32_desc(unsigned long lon
 // common path is kept short (packed 16-bit operations, loops instead of unrolled sequences), and
 // everything rare sits in functions of its own that are not inlined.
 
-// k-th largest of a slot's per-thread keys (lane l owns tkey[16 l .. 16 l + 16)): two 8-bit radix
-// passes over a shared histogram.  1 <= k <= 512.  Rare: only when the maxima spread over more
-// than 256 key values.
-__device__ __noinline__ uint32_t warp_kth_largest16(const uint16_t* tkey, int k, int* hist) {
-    const int lane = threadIdx.x & 31;
-    uint32_t prefix = 0;
-    int need = k;
-    for (int pass = 1; pass >= 0; --pass) {
-        for (int j = 0; j < 8; ++j) hist[lane * 8 + j] = 0;
-        __syncwarp();
-        for (int j = 0; j < kPerLane; ++j) {
-            const uint32_t key = tkey[lane * kPerLane + j];
-            if (pass == 1 || (key >> 8) == prefix) atomicAdd(&hist[(key >> (8 * pass)) & 255u], 1);
-        }
-        __syncwarp();
-        int c[8], mine = 0;
-        for (int j = 0; j < 8; ++j) { c[j] = hist[lane * 8 + j]; mine += c[j]; }
-        int incl = mine;                                   // suffix sums over lanes from the top
-        for (int o = 1; o < 32; o <<= 1) {
-            const int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
-            if (lane + o < 32) incl += u;
-        }
-        const int above = incl - mine;
-        const bool here = above < need && need <= incl;
-        int bin = 0, nd = 0;
-        if (here) {
-            int a = above, bb = 7;
-            while (bb > 0 && a + c[bb] < need) { a += c[bb]; --bb; }
-            bin = lane * 8 + bb; nd = need - a;
-        }
-        const int src = __ffs(__ballot_sync(0xFFFFFFFFu, here)) - 1;
-        bin = __shfl_sync(0xFFFFFFFFu, bin, src);
-        need = __shfl_sync(0xFFFFFFFFu, nd, src);
-        prefix = pass == 1 ? (uint32_t)bin : ((prefix << 8) | (uint32_t)bin);
-        __syncwarp();
-    }
-    return prefix;
-}
-
 // Exact path for one row by one warp: radix select on the 16-bit keys, ordered tie handling,
 // fp64 sum.  Leaves exactly kk candidates in f.cand and returns the row maximum and sum.
 __device__ __noinline__ void row_exact_warp(FinScratch& f, const uint16_t* row, int V, int kk, double& m_out, double& S_out) {
@@ -416,52 +377,28 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
     }
     const int myE = slot.warpE[lane >> 1];
     const int emax = __reduce_max_sync(0xFFFFFFFFu, myE);
-    uint32_t mk = kw[0];
+    uint32_t lane_mk = kw[0];
 #pragma unroll
-    for (int q = 1; q < kPerLane / 2; ++q) mk = __vmaxu2(mk, kw[q]);
-    mk = __reduce_max_sync(0xFFFFFFFFu, max(mk & 0xFFFFu, mk >> 16));
+    for (int q = 1; q < kPerLane / 2; ++q) lane_mk = __vmaxu2(lane_mk, kw[q]);
+    const uint32_t mk = __reduce_max_sync(0xFFFFFFFFu, max(lane_mk & 0xFFFFu, lane_mk >> 16));
 
-    // tau: the kk-th largest per-thread maximum.  The maxima of a row lie close together, so a
-    // histogram with one bin per key value over the 256 values below the largest usually holds kk
-    // of them (and spreads the shared-memory atomics); otherwise two generic radix passes.
-    uint32_t tau_key;
+    // tau: the kk-th largest of the 32 lanes' maxima (each the largest of 16 per-thread maxima).  That
+    // is at most the kk-th largest per-thread maximum, hence at most the row's kk-th largest logit, so
+    // every winner still lives in a thread whose maximum is >= tau; a few more threads than kk get
+    // flagged, and in exchange tau takes sixteen ballots instead of a histogram over 512 keys.
+    // (kk <= 32 always; with fewer than kk finite lane maxima tau is -inf and the row goes the exact way.)
+    uint32_t tau_key = 0;
     {
-        const uint32_t base = mk > 255u ? mk - 255u : 0u;
-        uint4* hp = reinterpret_cast<uint4*>(&f.hist[lane * 8]);
-        hp[0] = make_uint4(0, 0, 0, 0); hp[1] = make_uint4(0, 0, 0, 0);
-        __syncwarp();
+        const uint32_t lane_max = max(lane_mk & 0xFFFFu, lane_mk >> 16);
+        unsigned cand = 0xFFFFFFFFu;                       // lanes whose maximum matches tau's bits so far
+        int need = kk;
 #pragma unroll 1
-        for (int q = 0; q < kPerLane; ++q) {               // (keys from the slot again: a loop, not sixteen copies)
-            const uint32_t key = slot.tkey[lane * kPerLane + q];
-            if (key >= base) atomicAdd(&f.hist[key - base], 1);
+        for (int bit = 15; bit >= 0; --bit) {
+            const unsigned ones = __ballot_sync(0xFFFFFFFFu, (lane_max >> bit) & 1u) & cand;
+            const int c = __popc(ones);
+            if (c >= need) { tau_key |= 1u << bit; cand = ones; }
+            else { need -= c; cand &= ~ones; }
         }
-        __syncwarp();
-        const uint4 c0 = hp[0], c1 = hp[1];
-        const int c[8] = {(int)c0.x, (int)c0.y, (int)c0.z, (int)c0.w, (int)c1.x, (int)c1.y, (int)c1.z, (int)c1.w};
-        const int mine = ((c[0] + c[1]) + (c[2] + c[3])) + ((c[4] + c[5]) + (c[6] + c[7]));
-        int incl = mine;                                   // suffix sums over lanes from the top
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
-            if (lane + o < 32) incl += u;
-        }
-        const int above = incl - mine;
-        const bool here = above < kk && kk <= incl;
-        int bin = -1;
-        if (here) {
-            int a = above;
-#pragma unroll
-            for (int b = 7; b >= 0; --b) {                 // highest bin whose suffix count reaches kk
-                if (bin < 0) {
-                    if (a + c[b] >= kk) bin = lane * 8 + b;
-                    else a += c[b];
-                }
-            }
-        }
-        const unsigned hm = __ballot_sync(0xFFFFFFFFu, here);
-        __syncwarp();
-        if (hm) tau_key = base + (uint32_t)__shfl_sync(0xFFFFFFFFu, bin, __ffs(hm) - 1);
-        else tau_key = warp_kth_largest16(slot.tkey, kk, f.hist);
     }
     bool exact = tau_key <= kOrdNegInf || emax >= kExpLimit || emax <= -kExpLimit;
 
