@@ -422,11 +422,14 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
         eq += key == thr ? 1 : 0;
     }
     int total_eq, total;
-    const int eq_before = team_excl_scan(eq, s.scan_a, tw, total_eq);
-    if (dirty >= 0) { s.thist[dirty][tt] = 0; s.thist[dirty][tt + kTeam] = 0; }     // everyone is past the last pass
-    int eq_take = need_eq - eq_before;
-    eq_take = eq_take < 0 ? 0 : (eq_take > eq ? eq : eq_take);
+    int eq_take = 0;
+    if (need_eq > 0) {                                     // (the same for all warps) ties at the threshold: lowest indices first
+        const int eq_before = team_excl_scan(eq, s.scan_a, tw, total_eq);
+        eq_take = need_eq - eq_before;
+        eq_take = eq_take < 0 ? 0 : (eq_take > eq ? eq : eq_take);
+    }
     int pos = team_excl_scan(gt + eq_take, s.scan_b, tw, total);
+    if (dirty >= 0) { s.thist[dirty][tt] = 0; s.thist[dirty][tt + kTeam] = 0; }     // everyone is past the last pass
     #pragma unroll 1
     for (int i = lo; i < hi; ++i) {
         const unsigned long long key = s.keys[i];
