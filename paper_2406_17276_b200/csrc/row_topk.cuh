@@ -37,6 +37,7 @@ constexpr int kCandCap = 128;                      // candidate list capacity pe
 constexpr int kMaxFlag = 64;                       // flagged threads the fast finisher accepts
 constexpr int kDesc = 4;                           // rows a CTA may hold between ticket and descriptor read
 constexpr int kDescRing = 16;                      // descriptors kept: a row's lives until its finisher has copied it
+constexpr int kLaneTauMaxK = 16;                   // largest k for which the finisher's threshold comes from the lane maxima
 constexpr int kPerLane = kConsumers / 32;          // per-thread results one finisher lane handles (16)
 
 constexpr float kLog2e = 1.44269504088896340736f;
@@ -254,6 +255,80 @@ __device__ __forceinline__ unsigned long long warp_sort32_desc(unsigned long lon
 // common path is kept short (packed 16-bit operations, loops instead of unrolled sequences), and
 // everything rare sits in functions of its own that are not inlined.
 
+// k-th largest of a slot's per-thread keys (lane l owns tkey[16 l .. 16 l + 16)): two 8-bit radix
+// passes over a shared histogram.  1 <= k <= 512.  Rare: only when the maxima spread over more
+// than 256 key values.
+__device__ __noinline__ uint32_t warp_kth_largest16(const uint16_t* tkey, int k, int* hist) {
+    const int lane = threadIdx.x & 31;
+    uint32_t prefix = 0;
+    int need = k;
+    for (int pass = 1; pass >= 0; --pass) {
+        for (int j = 0; j < 8; ++j) hist[lane * 8 + j] = 0;
+        __syncwarp();
+        for (int j = 0; j < kPerLane; ++j) {
+            const uint32_t key = tkey[lane * kPerLane + j];
+            if (pass == 1 || (key >> 8) == prefix) atomicAdd(&hist[(key >> (8 * pass)) & 255u], 1);
+        }
+        __syncwarp();
+        int c[8], mine = 0;
+        for (int j = 0; j < 8; ++j) { c[j] = hist[lane * 8 + j]; mine += c[j]; }
+        int incl = mine;                                   // suffix sums over lanes from the top
+        for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
+            if (lane + o < 32) incl += u;
+        }
+        const int above = incl - mine;
+        const bool here = above < need && need <= incl;
+        int bin = 0, nd = 0;
+        if (here) {
+            int a = above, bb = 7;
+            while (bb > 0 && a + c[bb] < need) { a += c[bb]; --bb; }
+            bin = lane * 8 + bb; nd = need - a;
+        }
+        const int src = __ffs(__ballot_sync(0xFFFFFFFFu, here)) - 1;
+        bin = __shfl_sync(0xFFFFFFFFu, bin, src);
+        need = __shfl_sync(0xFFFFFFFFu, nd, src);
+        prefix = pass == 1 ? (uint32_t)bin : ((prefix << 8) | (uint32_t)bin);
+        __syncwarp();
+    }
+    return prefix;
+}
+
+// The kk-th largest of a slot's 512 per-thread maxima, exactly: a histogram with one bin per key
+// value over the 256 values below the largest usually holds kk of them (the maxima of a row lie close
+// together); otherwise two generic radix passes.  Used when kk is too large for the lanes' maxima to
+// give a useful bound (see finish_row_warp).
+__device__ __noinline__ uint32_t tau_from_histogram(FinScratch& f, const uint16_t* tkey, uint32_t mk, int kk) {
+    const int lane = threadIdx.x & 31;
+    const uint32_t base = mk > 255u ? mk - 255u : 0u;
+    for (int j = 0; j < 8; ++j) f.hist[lane * 8 + j] = 0;
+    __syncwarp();
+    for (int q = 0; q < kPerLane; ++q) {
+        const uint32_t key = tkey[lane * kPerLane + q];
+        if (key >= base) atomicAdd(&f.hist[key - base], 1);
+    }
+    __syncwarp();
+    int c[8], mine = 0;
+    for (int j = 0; j < 8; ++j) { c[j] = f.hist[lane * 8 + j]; mine += c[j]; }
+    int incl = mine;                                   // suffix sums over lanes from the top
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
+        if (lane + o < 32) incl += u;
+    }
+    const int above = incl - mine;
+    const bool here = above < kk && kk <= incl;
+    int bin = 0;
+    if (here) {
+        int a = above, bb = 7;
+        while (bb > 0 && a + c[bb] < kk) { a += c[bb]; --bb; }
+        bin = lane * 8 + bb;
+    }
+    const unsigned hm = __ballot_sync(0xFFFFFFFFu, here);
+    __syncwarp();
+    if (hm) return base + (uint32_t)__shfl_sync(0xFFFFFFFFu, bin, __ffs(hm) - 1);
+    return warp_kth_largest16(tkey, kk, f.hist);
+}
+
 // Exact path for one row by one warp: radix select on the 16-bit keys, ordered tie handling,
 // fp64 sum.  Leaves exactly kk candidates in f.cand and returns the row maximum and sum.
 __device__ __noinline__ void row_exact_warp(FinScratch& f, const uint16_t* row, int V, int kk, double& m_out, double& S_out) {
@@ -386,9 +461,13 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
     // is at most the kk-th largest per-thread maximum, hence at most the row's kk-th largest logit, so
     // every winner still lives in a thread whose maximum is >= tau; a few more threads than kk get
     // flagged, and in exchange tau takes sixteen ballots instead of a histogram over 512 keys.
-    // (kk <= 32 always; with fewer than kk finite lane maxima tau is -inf and the row goes the exact way.)
+    // With fewer than kk finite lane maxima tau is -inf and the row goes the exact way.  The bound gets
+    // loose as kk approaches the 32 lanes (about 32 ln(32 / (32 - kk)) threads are flagged), so beyond
+    // kLaneTauMaxK the exact kk-th largest per-thread maximum is used instead.
     uint32_t tau_key = 0;
-    {
+    if (kk > kLaneTauMaxK) {
+        tau_key = tau_from_histogram(f, slot.tkey, mk, kk);
+    } else {
         const uint32_t lane_max = max(lane_mk & 0xFFFFu, lane_mk >> 16);
         unsigned cand = 0xFFFFFFFFu;                       // lanes whose maximum matches tau's bits so far
         int need = kk;
