@@ -408,9 +408,9 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
     for (int i = tt * 2; i < N; i += 2 * kTeam) *reinterpret_cast<uint4*>(&j.cand_phat[i]) = make_uint4(0, 0, 0, 0);
     #pragma unroll 1
     for (int i = tt * 4; i < N; i += 4 * kTeam) *reinterpret_cast<uint4*>(&j.cand_tok[i]) = make_uint4(0, 0, 0, 0);
-    unsigned long long thr;
-    int need_eq;
-    const int dirty = team_radix_select(s, N, nl, tt, ko, ka, thr, need_eq);
+    unsigned long long thr = 0ull;                         // with no more candidates than wanted, all of them (key > 0) are taken
+    int need_eq = 0, dirty = -1;
+    if (nl < nvalid) dirty = team_radix_select(s, N, nl, tt, ko, ka, thr, need_eq);
     // ordered compaction: thread tt owns a contiguous stretch of candidates
     const int per = (N + kTeam - 1) / kTeam;
     const int lo = min(tt * per, N), hi = min(lo + per, N);

@@ -118,3 +118,22 @@ def test_argument_checks_return_status_codes():
     with pytest.raises(binding.OptTreeError) as e:
         ot.build(tab, torch.zeros(2, dtype=torch.int32, device="cuda"), float("nan"))
     assert e.value.code == binding.ERR_INVALID_ARG
+
+
+def test_exact_ties_are_broken_by_index():
+    """Every row gives k tokens the same logit and masks the rest, so every child has probability
+    exactly 1/k, all candidates of a layer have the same path value, and the selection is decided by
+    the tie rules alone (depth, then candidate index)."""
+    B, V, H, n, k, D = 4, 2048, 64, 64, 10, 6
+    w = synth.Workload("ties", B, V, n, k, D, 3.0, 1.1, 0.0, H=H, seed=5)
+    rng = np.random.default_rng(11)
+    ld = np.full((H, V), 0xFF80, np.uint16)                       # -inf
+    for h in range(H):
+        ld[h, rng.choice(V, k, replace=False)] = 0x3F80           # 1.0 in bf16
+    ot = binding.OptTree(V, H, n, k, D, B)
+    d = dev_table(ld)
+    roots = synth.root_tokens(B, V, 3)
+    for delta in (NEG_INF, 0.05):
+        g = gpu_step(ot, d, d, roots, delta)
+        o, st = _compare.compare_step(w, ld, ld, roots, delta, g)
+        assert st["exact"] == B and st["near_tie"] == 0, st
