@@ -246,6 +246,48 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
+def run_rows(args):
+    """The row step alone (fused softmax + top-k of Algorithm 1's expansion) over a list of rows
+    larger than L2: its own roofline line.  Not the benchmark's metric; one GPU."""
+    import torch
+    from paper_2406_17276_b200 import binding, build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    build.build()
+    w = synth.WORKLOADS[args.workload]
+    ld, _ = synth.make_tables(w)
+    d_ld = torch.from_numpy(ld.view(np.int16)).cuda()
+    ot = binding.OptTree(w.V, w.H, w.n, w.k, w.max_depth, w.batch)
+    nrows = args.rows
+    rows = torch.from_numpy(np.random.default_rng(w.seed).integers(0, w.H, nrows).astype(np.int32)).cuda()
+    for _ in range(max(3, args.warmup)):
+        ot.row_softmax_topk(d_ld, rows)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0); sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        ot.row_softmax_topk(d_ld, rows)
+    e1.record(); torch.cuda.synchronize()
+    clocks = sampler.result()
+    if ot.device_status() != 0:
+        raise SystemExit(f"bench.py: device status {ot.device_status()}")
+    ms = e0.elapsed_time(e1) / args.steps
+    peak, peak_kind = _peaks()
+    algo = 2.0 * w.V * nrows
+    achieved = algo / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "rows_per_s", "value": nrows / (ms * 1e-3), "unit": "rows/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{w.name}: row step alone, {nrows} random rows of V={w.V}, k={w.k}, H={w.H} bf16 table",
+                   "l2": "the 262 MB table is larger than L2; rows repeat across the list"},
+        "clocks": clocks, "gpu_launches": args.steps,
+        "roofline": {"bound": "hbm", "kernel": "row_topk_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": algo, "traffic": None},
+    }), flush=True)
+
+
 def cpu_baseline(w, ld, lt, steps, batch=None):
     """The oracle as it stands, single thread, un-memoised, on a bounded sample of the workload."""
     import oracle
@@ -294,9 +336,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu dram bytes per build call to report in roofline.traffic (default: the recorded capture, if the kernel sources are unchanged)")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="time the row step alone over this many rows instead of whole steps (its own roofline line)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.rows > 0:
+        run_rows(args)
     else:
         run_cuda(args)
 
