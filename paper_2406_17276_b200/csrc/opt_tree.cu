@@ -273,7 +273,8 @@ struct BuildSink {
             team_sync();
             const LayerJob j = ls.job;
             if (j.kind == 0) return;
-            select_layer_team(ls, j, tt, w.status);
+            if (j.fsize * j.k <= 1024) select_layer_team(ls, j, tt, w.status);
+            else select_layer_team_big(ls, j, tt, w.status);
         }
     }
     __device__ void layer_follow(LayerScratch& ls) {
@@ -309,20 +310,20 @@ struct BuildSink {
                     stage_layer_candidates(ls, sw, fsize, p.k);
                     unsigned g0 = 0;
                     if (early) g0 = reserve_layer(nl);        // the rows' numbers, while the candidates load
-                    if (fsize * p.k <= 1024) {
+                    {
+                        const bool small = fsize * p.k <= 1024;    // the candidates fit the shared-memory staging
                         if (lane == 0) {
                             LayerJob& j = ls.job;
                             j.kind = 1; j.d = d; j.fsize = fsize; j.n = p.n; j.k = p.k; j.kk = p.kk;
                             j.cand_phat = sw.cand_phat; j.cand_tok = sw.cand_tok;
                             j.T_tok = sw.T_tok; j.T_par = sw.T_par; j.T_phat = sw.T_phat;
                         }
-                        cp_async_wait_all();                  // the staged candidates are in shared memory
+                        if (small) cp_async_wait_all();       // the staged candidates are in shared memory
                         __syncwarp();
                         team_sync();                          // ... and, with the job, visible to the assistants
                         const LayerJob j = ls.job;
-                        select_layer_team(ls, j, lane, w.status);
-                    } else {
-                        select_layer_warp(ls, sw, d, fsize, p.n, p.k, p.kk, w.status);
+                        if (small) select_layer_team(ls, j, lane, w.status);
+                        else select_layer_team_big(ls, j, lane, w.status);
                     }
                     if (early) publish_layer(ls, b, d, nl, g0);
                     const bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta,

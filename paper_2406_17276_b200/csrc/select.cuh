@@ -1,5 +1,5 @@
-// K2 / K3 by one warp: layer selection (the n candidates of largest path value), running
-// E_sub(T, n), the loop test of Algorithm 1, and the scan-based tree packer.
+// K2 / K3: layer selection (the n candidates of largest path value) by the layer team, running
+// E_sub(T, n), the loop test of Algorithm 1 and the scan-based tree packer by the layer warp.
 //
 // Selection never sorts: an 8-pass radix select on the 64-bit keys finds the threshold of the
 // "need" largest, then an ordered compaction (ballot scans) emits the kept elements in index
@@ -108,44 +108,6 @@ __device__ int warp_compact_selected(KeyFn keyf, int N, unsigned long long thr, 
     return taken;
 }
 
-// The same selection, but every lane owns a contiguous stretch of `per` elements (lane l: indices
-// l*per .. l*per+per, cut at N), so that positions follow from one count per lane and one warp scan
-// instead of a ballot per 32 elements.  The kept indices go to idx[0..kept) first (a lane may own
-// many of them), then emit(pos, i) runs over the positions spread evenly over the lanes.  Returns
-// the number kept.  Whole warp.
-template <class KeyFn, class EmitFn>
-__device__ int warp_compact_selected_blocked(KeyFn keyf, int N, unsigned long long thr, int need_eq, int* idx, EmitFn emit) {
-    const int lane = threadIdx.x & 31;
-    const int per = (N + 31) >> 5;
-    const int lo = min(lane * per, N), hi = min(lo + per, N);
-    int gt = 0, eq = 0;
-#pragma unroll 4
-    for (int i = lo; i < hi; ++i) {
-        const unsigned long long key = keyf(i);
-        gt += key > thr ? 1 : 0;
-        eq += key == thr ? 1 : 0;
-    }
-    int total_eq, total;
-    const int eq_before = warp_excl_scan(eq, total_eq);
-    int eq_take = need_eq - eq_before;
-    eq_take = eq_take < 0 ? 0 : (eq_take > eq ? eq : eq_take);
-    int pos = warp_excl_scan(gt + eq_take, total);
-    if (gt + eq_take > 0) {
-        #pragma unroll 1
-        for (int i = lo; i < hi; ++i) {
-            const unsigned long long key = keyf(i);
-            bool take = key > thr;
-            if (key == thr && eq_take > 0) { take = true; --eq_take; }
-            if (take) idx[pos++] = i;
-        }
-    }
-    __syncwarp();
-    #pragma unroll 1
-    for (int q = lane; q < total; q += 32) emit(q, idx[q]);
-    __syncwarp();
-    return total;
-}
-
 // Per-sequence state and arrays in the workspace (device pointers already offset to the sequence).
 struct SeqWork {
     double* cand_phat;     // [n*k, padded to a multiple of 4, 16-byte aligned]  path values of this layer's candidates (Eq. 2), slot-major
@@ -168,7 +130,7 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
 };
 
 // Starts the asynchronous copies of a layer's candidates (path values and tokens) into the layer
-// warp's scratch; select_layer_warp waits for them.  Separate so that other round trips (the
+// warp's scratch; the layer warp waits for them before it starts the team.  Separate so that other round trips (the
 // mailbox reservations) can be in flight at the same time.
 __device__ __forceinline__ void stage_layer_candidates(LayerScratch& s, const SeqWork& w, int fsize, int k) {
     const int lane = threadIdx.x & 31;
@@ -180,100 +142,6 @@ __device__ __forceinline__ void stage_layer_candidates(LayerScratch& s, const Se
     for (int i = lane * 2; i < N; i += 64) cp_async_16(&s.keys[i], &gph[i]);
     #pragma unroll 1
     for (int i = lane * 4; i < N; i += 128) cp_async_16(&s.toks[i], &gtk[i]);
-}
-
-// Layer job, first half.  After all rows of layer d (1-based) of one sequence are expanded: the
-// next layer = the nl candidates of largest path value, stored in candidate-index order (nodes
-// gid0 .. gid0+nl of T; tokens and keys also left in s.ltok / s.lkeys).  Whole layer warp; s is its scratch; fsize = rows of the layer.  Returns nl.
-__device__ __noinline__ int select_layer_warp(LayerScratch& s, const SeqWork& w, int d, int fsize, int n, int k, int kk, int* status) {
-    const int lane = threadIdx.x & 31;
-    int* hist = s.hist;
-    const int N = fsize * k;
-    const int nvalid = fsize * kk;
-    const int nl = nvalid < n ? nvalid : n;
-    const int gid0 = (d - 1) * n;
-    unsigned long long thr;
-    int need_eq;
-    // Candidate words validate themselves (written by other SMs' finisher warps without a fence): top
-    // bit set = written; all ones = no such child.  A word not yet written is simply read again.
-    const unsigned long long* gph = reinterpret_cast<const unsigned long long*>(w.cand_phat);
-    const unsigned int* gtk = reinterpret_cast<const unsigned int*>(w.cand_tok);
-    auto wait_phat = [&](int i) -> unsigned long long {
-        unsigned long long x = ld_relaxed_u64(&gph[i]);
-        for (int t = 0; !(x >> 63) && t < (1 << 22); ++t) x = ld_relaxed_u64(&gph[i]);
-        if (!(x >> 63)) { set_status(status, kErrTimeout); x = ~0ull; }
-        return x;
-    };
-    auto wait_tok = [&](int i) -> int {
-        unsigned int x = ld_relaxed_u32(&gtk[i]);
-        for (int t = 0; !(x >> 31) && t < (1 << 22); ++t) x = ld_relaxed_u32(&gtk[i]);
-        if (!(x >> 31)) { set_status(status, kErrTimeout); x = ~0u; }
-        return x == ~0u ? -1 : (int)(x & 0x7FFFFFFFu);
-    };
-    auto key_of = [](unsigned long long x) -> unsigned long long { return x == ~0ull ? 0ull : (x & 0x7FFFFFFFFFFFFFFFull) + 1ull; };
-    unsigned long long ko = 0ull, ka = ~0ull;
-    if (N <= 1024) {
-        // Stage path values and tokens in shared memory with 16-byte asynchronous copies, so that all
-        // loads are in flight together (one round trip); then the keys in place.  The per-sequence
-        // candidate arrays are padded to a multiple of four entries, so reading the last vector whole
-        // stays inside them.
-        // (the copies were started by stage_layer_candidates)
-        cp_async_wait_all();
-        __syncwarp();
-#pragma unroll 4
-        for (int i = lane; i < N; i += 32) {
-            unsigned long long x = s.keys[i];
-            if (!(x >> 63)) x = wait_phat(i);
-            const unsigned long long key = key_of(x);
-            s.keys[i] = key;
-            if (key) { ko |= key; ka &= key; }
-            // a token word that was not yet there when it was staged must be fetched before the arrays are
-            // cleared: a store that lands late would otherwise be wiped out, or wipe out a later layer's word
-            const unsigned int t = (unsigned int)s.toks[i];
-            if (!(t >> 31)) { const int tok = wait_tok(i); s.toks[i] = tok < 0 ? -1 : (int)(0x80000000u | (unsigned int)tok); }
-        }
-        __syncwarp();
-        // the arrays are free for the next layer's rows once they are zero again
-        #pragma unroll 1
-        for (int i = lane * 2; i < N; i += 64) *reinterpret_cast<uint4*>(&w.cand_phat[i]) = make_uint4(0, 0, 0, 0);
-        #pragma unroll 1
-        for (int i = lane * 4; i < N; i += 128) *reinterpret_cast<uint4*>(&w.cand_tok[i]) = make_uint4(0, 0, 0, 0);
-        auto skey = [&](int i) -> unsigned long long { return s.keys[i]; };
-        warp_radix_select(skey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
-        warp_compact_selected_blocked(skey, N, thr, need_eq, s.gids, [&](int pos, int i) {
-            const unsigned int t = (unsigned int)s.toks[i];                  // staged word, validated above
-            const int tok = t == ~0u ? -1 : (int)(t & 0x7FFFFFFFu);
-            w.T_tok[gid0 + pos] = tok;
-            s.ltok[pos] = tok;
-            w.T_par[gid0 + pos] = i / k;
-            w.T_phat[gid0 + pos] = __longlong_as_double((long long)(s.keys[i] - 1ull));
-            s.lkeys[pos] = s.keys[i];
-        });
-    } else {
-        auto gkey = [&](int i) -> unsigned long long { return key_of(wait_phat(i)); };
-        #pragma unroll 1
-        for (int i = lane; i < N; i += 32) {
-            const unsigned long long key = gkey(i);
-            if (key) { ko |= key; ka &= key; }
-        }
-        warp_radix_select(gkey, N, nl, hist, warp_or_u64(ko), warp_and_u64(ka), thr, need_eq);
-        warp_compact_selected(gkey, N, thr, need_eq, [&](int pos, int i) {
-            const unsigned long long key = gkey(i);
-            const int tok = wait_tok(i);
-            w.T_tok[gid0 + pos] = tok;
-            s.ltok[pos] = tok;
-            w.T_par[gid0 + pos] = i / k;
-            w.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
-            s.lkeys[pos] = key;
-        });
-        __syncwarp();
-        #pragma unroll 1
-        for (int i = lane * 2; i < N; i += 64) *reinterpret_cast<uint4*>(&w.cand_phat[i]) = make_uint4(0, 0, 0, 0);
-        #pragma unroll 1
-        for (int i = lane * 4; i < N; i += 128) *reinterpret_cast<uint4*>(&w.cand_tok[i]) = make_uint4(0, 0, 0, 0);
-    }
-    __syncwarp();
-    return nl;
 }
 
 // A candidate word that was not there yet when it was looked at is read again until it is (bounded).
@@ -314,8 +182,14 @@ __device__ __forceinline__ int team_excl_scan(int v, int* wtot, int tw, int& tot
 // arrays that are all zero on entry: pass p counts into array p % 3 and clears the one pass p-1
 // read, so one barrier per pass is enough.  Returns the array that is left non-zero (the caller
 // clears it after its next barrier), or -1.
-__device__ int team_radix_select(LayerScratch& s, int N, int need, int tt, unsigned long long key_or, unsigned long long key_and,
-                                 unsigned long long& thr, int& need_eq) {
+// kGlobal: the keys are not staged; they are read from the candidate words gw[0..N) in global memory
+// (all written: the caller has looked at every one), eight loads in flight per thread.
+__device__ __forceinline__ unsigned long long key_of_word(unsigned long long x) {
+    return x == ~0ull ? 0ull : (x & 0x7FFFFFFFFFFFFFFFull) + 1ull;
+}
+template <bool kGlobal>
+__device__ int team_radix_select(LayerScratch& s, const unsigned long long* gw, int N, int need, int tt, unsigned long long key_or,
+                                 unsigned long long key_and, unsigned long long& thr, int& need_eq) {
     const int lane = threadIdx.x & 31;
     const unsigned long long diff = key_or ^ key_and;
     if (diff == 0ull) { thr = key_or; need_eq = need; return -1; }       // all elements equal
@@ -326,11 +200,26 @@ __device__ int team_radix_select(LayerScratch& s, int N, int need, int tt, unsig
         const int wbits = top < 8 ? top : 8, shift = top - wbits;
         const unsigned int dmask = (1u << wbits) - 1u;
         int* hist = s.thist[pass % 3];
-        #pragma unroll 1
-        for (int i = tt; i < N; i += kTeam) {
-            const unsigned long long key = s.keys[i];
-            const bool match = key != 0ull && (top == 64 || (key >> top) == (prefix >> top));
-            if (match) atomicAdd(&hist[(int)((unsigned int)(key >> shift) & dmask)], 1);
+        if (!kGlobal) {
+            #pragma unroll 1
+            for (int i = tt; i < N; i += kTeam) {
+                const unsigned long long key = s.keys[i];
+                const bool match = key != 0ull && (top == 64 || (key >> top) == (prefix >> top));
+                if (match) atomicAdd(&hist[(int)((unsigned int)(key >> shift) & dmask)], 1);
+            }
+        } else {
+            #pragma unroll 1
+            for (int i0 = tt; i0 < N; i0 += 8 * kTeam) {
+                unsigned long long x[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) x[u] = i0 + u * kTeam < N ? ld_relaxed_u64(&gw[i0 + u * kTeam]) : ~0ull;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const unsigned long long key = key_of_word(x[u]);
+                    const bool match = key != 0ull && (top == 64 || (key >> top) == (prefix >> top));
+                    if (match) atomicAdd(&hist[(int)((unsigned int)(key >> shift) & dmask)], 1);
+                }
+            }
         }
         team_sync();
         int c[8], mine = 0;
@@ -410,7 +299,7 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
     for (int i = tt * 4; i < N; i += 4 * kTeam) *reinterpret_cast<uint4*>(&j.cand_tok[i]) = make_uint4(0, 0, 0, 0);
     unsigned long long thr = 0ull;                         // with no more candidates than wanted, all of them (key > 0) are taken
     int need_eq = 0, dirty = -1;
-    if (nl < nvalid) dirty = team_radix_select(s, N, nl, tt, ko, ka, thr, need_eq);
+    if (nl < nvalid) dirty = team_radix_select<false>(s, nullptr, N, nl, tt, ko, ka, thr, need_eq);
     // ordered compaction: thread tt owns a contiguous stretch of candidates
     const int per = (N + kTeam - 1) / kTeam;
     const int lo = min(tt * per, N), hi = min(lo + per, N);
@@ -451,6 +340,93 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
     return nl;
 }
 
+// The team's selection for layers with more candidates than the shared-memory staging holds
+// (1024 < N <= n*k): the same steps, but every sweep reads the candidate words from global memory
+// (they sit in L2), a thread's loads eight at a time.  The candidate arrays are cleared at the end.
+__device__ __noinline__ int select_layer_team_big(LayerScratch& s, const LayerJob& j, int tt, int* status) {
+    const int lane = threadIdx.x & 31, tw = tt >> 5;
+    const int N = j.fsize * j.k;
+    const int nvalid = j.fsize * j.kk;
+    const int nl = nvalid < j.n ? nvalid : j.n;
+    const int gid0 = (j.d - 1) * j.n;
+    const unsigned long long* gph = reinterpret_cast<const unsigned long long*>(j.cand_phat);
+    const unsigned int* gtk = reinterpret_cast<const unsigned int*>(j.cand_tok);
+    unsigned long long ko = 0ull, ka = ~0ull;
+    #pragma unroll 1
+    for (int i0 = tt; i0 < N; i0 += 8 * kTeam) {
+        unsigned long long x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) x[u] = i0 + u * kTeam < N ? ld_relaxed_u64(&gph[i0 + u * kTeam]) : ~0ull;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (!(x[u] >> 63)) x[u] = poll_phat_word(&gph[i0 + u * kTeam], status);      // not written yet: read again
+            const unsigned long long key = key_of_word(x[u]);
+            if (key) { ko |= key; ka &= key; }
+        }
+    }
+    ko = warp_or_u64(ko); ka = warp_and_u64(ka);
+    if (lane == 0) { s.red_or[tw] = ko; s.red_and[tw] = ka; }
+    team_sync();
+    ko = 0ull; ka = ~0ull;
+#pragma unroll
+    for (int q = 0; q < kTeamWarps; ++q) { ko |= s.red_or[q]; ka &= s.red_and[q]; }
+    unsigned long long thr = 0ull;
+    int need_eq = 0, dirty = -1;
+    if (nl < nvalid) dirty = team_radix_select<true>(s, gph, N, nl, tt, ko, ka, thr, need_eq);
+    // ordered compaction: thread tt owns a contiguous stretch of candidates (a multiple of 8 long)
+    const int per = (((N + kTeam - 1) / kTeam) + 7) & ~7;
+    const int lo = min(tt * per, N), hi = min(lo + per, N);
+    int gt = 0, eq = 0;
+    #pragma unroll 1
+    for (int i0 = lo; i0 < hi; i0 += 8) {
+        unsigned long long x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) x[u] = i0 + u < hi ? ld_relaxed_u64(&gph[i0 + u]) : ~0ull;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const unsigned long long key = key_of_word(x[u]);
+            gt += key > thr ? 1 : 0;
+            eq += (key == thr && key != 0ull) ? 1 : 0;
+        }
+    }
+    int total_eq, total;
+    int eq_take = 0;
+    if (need_eq > 0) {
+        const int eq_before = team_excl_scan(eq, s.scan_a, tw, total_eq);
+        eq_take = need_eq - eq_before;
+        eq_take = eq_take < 0 ? 0 : (eq_take > eq ? eq : eq_take);
+    }
+    int pos = team_excl_scan(gt + eq_take, s.scan_b, tw, total);
+    if (dirty >= 0) { s.thist[dirty][tt] = 0; s.thist[dirty][tt + kTeam] = 0; }
+    if (gt + eq_take > 0) {
+        #pragma unroll 1
+        for (int i = lo; i < hi; ++i) {
+            const unsigned long long key = key_of_word(ld_relaxed_u64(&gph[i]));
+            bool take = key > thr;
+            if (key == thr && key != 0ull && eq_take > 0) { take = true; --eq_take; }
+            if (take) {
+                unsigned int t32 = ld_relaxed_u32(&gtk[i]);
+                if (!(t32 >> 31)) t32 = poll_tok_word(&gtk[i], status);
+                const int tok = t32 == ~0u ? -1 : (int)(t32 & 0x7FFFFFFFu);
+                j.T_tok[gid0 + pos] = tok;
+                s.ltok[pos] = tok;
+                j.T_par[gid0 + pos] = i / j.k;
+                j.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
+                s.lkeys[pos] = key;
+                ++pos;
+            }
+        }
+    }
+    if (total != nl) set_status(status, kErrInternal);
+    team_sync();                                           // everyone has read what it needs: the arrays can be cleared
+    #pragma unroll 1
+    for (int i = tt * 2; i < N; i += 2 * kTeam) *reinterpret_cast<uint4*>(&j.cand_phat[i]) = make_uint4(0, 0, 0, 0);
+    #pragma unroll 1
+    for (int i = tt * 4; i < N; i += 4 * kTeam) *reinterpret_cast<uint4*>(&j.cand_tok[i]) = make_uint4(0, 0, 0, 0);
+    team_sync();
+    return nl;
+}
+
 // Once per sequence, when it is finished: T_opt = the running top-n (s.rsel / s.vals, already in
 // (depth, parent's index, sibling rank) order), packed with parent indices.
 __device__ __noinline__ void pack_tree_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nR, int n, int max_depth,
@@ -483,7 +459,7 @@ __device__ __noinline__ void pack_tree_warp(LayerScratch& s, const SeqWork& w, c
 }
 
 // Layer job, second half: the running top-n and E_sub(T, n) with the new layer (left in s by
-// select_layer_warp), the loop test of Algorithm 1, and the packed tree if the sequence is
+// the selection), the loop test of Algorithm 1, and the packed tree if the sequence is
 // finished.  All layers of a sequence are handled by the same warp, in order.  Returns true if the
 // sequence continues with layer d+1, false if it is finished (outputs written).
 __device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
