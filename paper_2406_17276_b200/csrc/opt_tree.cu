@@ -349,7 +349,7 @@ struct BuildSink {
     }
 };
 
-// Algorithm 1 for a whole batch in one launch: persistent CTAs pull rows from the queue; layers
+// Algorithm 1 for a whole batch in one launch: persistent CTAs take rows from their mailboxes; layers
 // of different sequences overlap freely because sequences never exchange data.
 __global__ void __launch_bounds__(kThreads)
 build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, opt_tree_out out) {

@@ -1,7 +1,7 @@
 // The persistent, warp-specialised row pipeline of one CTA.
 //
 //   fetcher warp    asks a Source for row descriptors, several at a time and ahead of the
-//                   consumers, so that the latency of obtaining work (a queue pop, an index load)
+//                   consumers, so that the latency of obtaining work (a mailbox entry, an index load)
 //                   is hidden, and hands them on in the order in which they become known;
 //   issuer warp     streams each described row's chunks into the ring (bulk async copies) as
 //                   stages are handed back;
@@ -19,7 +19,9 @@
 // (g / kStages)-th use of that stage, which fixes every mbarrier parity; likewise row r uses
 // descriptor r % kDesc and slot r % kSlots.  Every row has the same number of chunks (V is fixed).
 // All waits are bounded (common.cuh); a role that times out leaves its loop, and the others then
-// time out on it in turn, so the CTA always ends.
+// time out on it in turn, so the CTA always ends.  The one wait without a clock is the layer team's
+// barrier: the assistants sit there between jobs, and the layer warp, whose own waits are all
+// bounded, reaches it however it leaves its loop (it then posts a last job that sends them home).
 #pragma once
 
 #include "row_topk.cuh"
@@ -39,7 +41,7 @@ __device__ __forceinline__ void pipeline_init(CtaSmem& s) {
 }
 
 // ---- fetcher warp ------------------------------------------------------------------------------
-// Obtaining a row costs global-memory round trips (a queue pop and its item, an index load) that
+// Obtaining a row costs global-memory round trips (a mailbox entry, an index load) that
 // take about as long as streaming the row, so kFetchLanes lanes hold one ticket each and poll
 // concurrently; the warp stays converged in one polling loop so that the lanes' round trips
 // overlap.  Rows are handed on in the order in which they become known (the a-th known row goes to
