@@ -157,8 +157,10 @@ int opt_tree_row_softmax_topk(opt_tree_ctx *ctx, const void *logits_bf16, const 
 /* One whole decoding step (build, mask, verify) with HOST buffers: copies root_token and
  * base_pos to the device, runs the three stages, copies every output back and synchronises the
  * stream before returning.  The logit tables stay on the device (they stand in for the models).
- * Host buffers should be pinned for the copies to be asynchronous.  Any output pointer may be
- * NULL to skip its copy; shapes are those of opt_tree_out / opt_tree_mask / opt_tree_verify. */
+ * The inputs and the outputs cross the bus in one copy each, through pinned staging memory the
+ * context owns (so the caller's buffers need not be pinned); the staging is reused by every call,
+ * hence one call at a time per context.  Any output pointer may be NULL to skip it; shapes are
+ * those of opt_tree_out / opt_tree_mask / opt_tree_verify. */
 typedef struct {
     int32_t *token, *parent, *depth; double *phat;                 /* (host) [B][n] */
     int32_t *n_sel, *depth_reached; double *expected_len;          /* (host) [B] */

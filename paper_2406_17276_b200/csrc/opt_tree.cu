@@ -551,6 +551,10 @@ struct opt_tree_ctx {
     int grid;              // resident CTAs of the persistent kernels (SMs x occupancy)
     int mcap;
     int64_t launches;
+    // pinned host staging of opt_tree_step_host: the step's inputs and outputs cross the bus in one
+    // copy each and are spread to / gathered from the caller's arrays on the host
+    char* hstage;
+    size_t in_bytes, out_bytes;     // device ranges [h_root, end of h_base) and [o_token, end of o_next)
 };
 
 namespace {
@@ -631,7 +635,12 @@ int opt_tree_create(opt_tree_ctx** out, const opt_tree_config* cfg) {
         return OPT_TREE_ERR_CUDA;
     }
     ot::carve(*cfg, ctx->grid, static_cast<char*>(ctx->base), &ctx->ws);
-    if (cudaMemset(ctx->base, 0, ctx->bytes) != cudaSuccess) {
+    // (carve lays h_root, h_base out next to each other, and likewise o_token ... o_next)
+    ctx->in_bytes = (size_t)(reinterpret_cast<char*>(ctx->ws.h_base + cfg->max_batch) - reinterpret_cast<char*>(ctx->ws.h_root));
+    ctx->out_bytes = (size_t)(reinterpret_cast<char*>(ctx->ws.o_next + cfg->max_batch) - reinterpret_cast<char*>(ctx->ws.o_token));
+    ctx->hstage = nullptr;
+    if (cudaMemset(ctx->base, 0, ctx->bytes) != cudaSuccess ||
+        cudaHostAlloc(reinterpret_cast<void**>(&ctx->hstage), ctx->in_bytes + ctx->out_bytes, cudaHostAllocDefault) != cudaSuccess) {
         cudaGetLastError();
         cudaFree(ctx->base);
         delete ctx;
@@ -643,6 +652,7 @@ int opt_tree_create(opt_tree_ctx** out, const opt_tree_config* cfg) {
 
 int opt_tree_destroy(opt_tree_ctx* ctx) {
     if (!ctx) return OPT_TREE_ERR_INVALID_ARG;
+    if (ctx->hstage) cudaFreeHost(ctx->hstage);
     cudaError_t e = cudaFree(ctx->base);
     delete ctx;
     return e == cudaSuccess ? OPT_TREE_OK : OPT_TREE_ERR_CUDA;
@@ -702,22 +712,30 @@ int opt_tree_step_host(opt_tree_ctx* ctx, const void* draft, const void* target,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const ot::Workspace& w = ctx->ws;
     const size_t n = ctx->cfg.n, D = ctx->cfg.max_depth, W = (ctx->cfg.n + 63) / 64, Bz = B;
-    bool ok = cudaMemcpyAsync(w.h_root, root_host, Bz * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (base_host) ok = ok && cudaMemcpyAsync(w.h_base, base_host, Bz * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (!ok) return OPT_TREE_ERR_CUDA;
+    // inputs: one copy of the range that holds both device arrays
+    char* hin = ctx->hstage;
+    char* hout = ctx->hstage + ctx->in_bytes;
+    const char* din = reinterpret_cast<const char*>(w.h_root);
+    memcpy(hin, root_host, Bz * 4);
+    if (base_host) memcpy(hin + (reinterpret_cast<const char*>(w.h_base) - din), base_host, Bz * 4);
+    if (cudaMemcpyAsync(w.h_root, hin, ctx->in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return OPT_TREE_ERR_CUDA;
     opt_tree_out t = {w.o_token, w.o_parent, w.o_depth, w.o_phat, w.o_nsel, w.o_dreach, w.o_elen, nullptr};
     int rc = opt_tree_build(ctx, draft, w.h_root, B, delta, &t, stream);
     if (rc == OPT_TREE_OK) rc = opt_tree_mask(ctx, &t, B, base_host ? w.h_base : nullptr, w.o_mask, w.o_pos, stream);
     if (rc == OPT_TREE_OK) rc = opt_tree_verify(ctx, &t, target, w.h_root, B, w.o_alen, w.o_atok, w.o_anode, w.o_next, stream);
     if (rc != OPT_TREE_OK) return rc;
-#define OT_D2H(dst, src, bytes) if (ok && (dst)) ok = cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    OT_D2H(ho->token, w.o_token, Bz * n * 4) OT_D2H(ho->parent, w.o_parent, Bz * n * 4) OT_D2H(ho->depth, w.o_depth, Bz * n * 4)
-    OT_D2H(ho->phat, w.o_phat, Bz * n * 8) OT_D2H(ho->n_sel, w.o_nsel, Bz * 4) OT_D2H(ho->depth_reached, w.o_dreach, Bz * 4)
-    OT_D2H(ho->expected_len, w.o_elen, Bz * 8) OT_D2H(ho->mask, w.o_mask, Bz * n * W * 8) OT_D2H(ho->position_ids, w.o_pos, Bz * n * 4)
-    OT_D2H(ho->accept_len, w.o_alen, Bz * 4) OT_D2H(ho->accept_tokens, w.o_atok, Bz * (D + 1) * 4)
-    OT_D2H(ho->accept_nodes, w.o_anode, Bz * D * 4) OT_D2H(ho->next_root, w.o_next, Bz * 4)
-#undef OT_D2H
-    if (!ok || cudaStreamSynchronize(st) != cudaSuccess) return OPT_TREE_ERR_CUDA;
+    // outputs: one copy of the range that holds all result arrays, then each to the caller's array
+    const char* dout = reinterpret_cast<const char*>(w.o_token);
+    if (cudaMemcpyAsync(hout, dout, ctx->out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return OPT_TREE_ERR_CUDA;
+#define OT_OUT(dst, src, bytes) if (dst) memcpy((dst), hout + (reinterpret_cast<const char*>(src) - dout), (bytes));
+    OT_OUT(ho->token, w.o_token, Bz * n * 4) OT_OUT(ho->parent, w.o_parent, Bz * n * 4) OT_OUT(ho->depth, w.o_depth, Bz * n * 4)
+    OT_OUT(ho->phat, w.o_phat, Bz * n * 8) OT_OUT(ho->n_sel, w.o_nsel, Bz * 4) OT_OUT(ho->depth_reached, w.o_dreach, Bz * 4)
+    OT_OUT(ho->expected_len, w.o_elen, Bz * 8) OT_OUT(ho->mask, w.o_mask, Bz * n * W * 8) OT_OUT(ho->position_ids, w.o_pos, Bz * n * 4)
+    OT_OUT(ho->accept_len, w.o_alen, Bz * 4) OT_OUT(ho->accept_tokens, w.o_atok, Bz * (D + 1) * 4)
+    OT_OUT(ho->accept_nodes, w.o_anode, Bz * D * 4) OT_OUT(ho->next_root, w.o_next, Bz * 4)
+#undef OT_OUT
     return OPT_TREE_OK;
 }
 
