@@ -54,7 +54,10 @@ def test_full_size_configurations(name, steps):
 
 
 @pytest.mark.parametrize("n,k,D,B,V", [(1, 4, 5, 3, 512), (6, 1, 6, 3, 512), (256, 32, 20, 2, 4096), (5, 8, 3, 4, 8),
-                                       (7, 3, 4, 2, 12), (64, 10, 10, 1, 32000), (10, 10, 6, 5, 100)])
+                                       (7, 3, 4, 2, 12), (64, 10, 10, 1, 32000), (10, 10, 6, 5, 100),
+                                       # more sequences than CTAs (a layer warp follows several), and more than
+                                       # four per CTA (they are then followed in waves)
+                                       (8, 4, 4, 300, 512), (6, 3, 3, 700, 256)])
 def test_degenerate_and_maximum_sizes(n, k, D, B, V):
     w = synth.Workload("edge", B, V, n, k, D, 3.0, 1.1, 0.3, H=64, seed=n * 1000 + k)
     t = _run(w, [NEG_INF, 0.1], steps=2)
