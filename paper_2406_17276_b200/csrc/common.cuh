@@ -185,6 +185,11 @@ __device__ __forceinline__ bool mbar_wait_thread(unsigned long long* bar, uint32
     return true;
 }
 
+// --- programmatic dependent launch: a kernel launched "after" another in the same stream may be
+//     set up while its predecessor drains; nothing of the predecessor's may be read or overwritten
+//     before this returns (no effect in a kernel launched the ordinary way) ---
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // --- barrier of the layer team (named barrier 1; barrier 0 is the CTA's) ---
 __device__ __forceinline__ void team_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kTeam) : "memory"); }
 

@@ -165,6 +165,7 @@ __device__ __forceinline__ unsigned long long phat_word(double p) {
 // ------------------------------------------------------------------------------------------------
 // Clears the mailboxes, sends the root row of sequence b to CTA b % grid and resets the per-sequence state.
 __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restrict__ root_token) {
+    grid_dependency_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < p.grid * p.mcap) {
         const int c = i / p.mcap, j = i - c * p.mcap;
@@ -400,6 +401,7 @@ row_topk_kernel(Params p, const uint16_t* __restrict__ logits, const int32_t* __
 __global__ void __launch_bounds__(kSmallThreads)
 mask_kernel(const int32_t* __restrict__ parent, const int32_t* __restrict__ depth, const int32_t* __restrict__ n_sel,
             const int32_t* __restrict__ base_pos, int n, uint64_t* mask, int32_t* position_ids, int* status) {
+    grid_dependency_wait();
     const int b = blockIdx.x, i = threadIdx.x;
     if (i >= n) return;
     const int W = (n + 63) >> 6;
@@ -445,6 +447,7 @@ __global__ void __launch_bounds__(kSmallThreads)
 verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const int32_t* __restrict__ root_token,
               opt_tree_out tree, int32_t* accept_len, int32_t* accept_tokens, int32_t* accept_nodes, int32_t* next_root) {
     __shared__ VerifySmem s;
+    grid_dependency_wait();
     const int b = blockIdx.y, j = blockIdx.x, tid = threadIdx.x;
     const int ns = tree.n_sel[b];
     if (j > ns) return;
@@ -582,6 +585,18 @@ ot::Params make_params(const opt_tree_ctx* ctx, const void* table, float delta) 
     p.aligned = ((reinterpret_cast<uintptr_t>(table) & 15u) == 0 && (c.V % 8) == 0) ? 1 : 0;
     return p;
 }
+// Launches a kernel that may be set up while the kernel before it in the stream drains (every kernel of
+// this library waits for its predecessor before it touches global memory, see grid_dependency_wait).
+template <class... KArgs, class... Args>
+void launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 bool bad_tree(const opt_tree_out* t) {
     return !t || !t->token || !t->parent || !t->depth || !t->phat || !t->n_sel || !t->depth_reached || !t->expected_len;
 }
@@ -666,9 +681,9 @@ int opt_tree_build(opt_tree_ctx* ctx, const void* draft, const int32_t* root_tok
     ot::Params p = make_params(ctx, draft, delta);
     p.B = B;
     const long long init_threads = (long long)ctx->grid * ctx->mcap > B ? (long long)ctx->grid * ctx->mcap : B;
-    ot::init_build_kernel<<<(unsigned)((init_threads + 255) / 256), 256, 0, st>>>(ctx->ws, p, root_token);
-    ot::build_kernel<<<ctx->grid, ot::kThreads, sizeof(ot::CtaSmem), st>>>(
-        ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
+    launch_after(ot::init_build_kernel, dim3((unsigned)((init_threads + 255) / 256)), dim3(256), 0, st, ctx->ws, p, root_token);
+    launch_after(ot::build_kernel, dim3(ctx->grid), dim3(ot::kThreads), sizeof(ot::CtaSmem), st,
+                 ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
     ctx->launches += 2;
     return check_launch();
 }
@@ -676,8 +691,8 @@ int opt_tree_build(opt_tree_ctx* ctx, const void* draft, const int32_t* root_tok
 int opt_tree_mask(opt_tree_ctx* ctx, const opt_tree_out* tree, int32_t B, const int32_t* base_pos, uint64_t* mask,
                   int32_t* position_ids, void* stream) {
     if (!ctx || bad_tree(tree) || !mask || !position_ids || B < 1 || B > ctx->cfg.max_batch) return OPT_TREE_ERR_INVALID_ARG;
-    ot::mask_kernel<<<B, ot::kSmallThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        tree->parent, tree->depth, tree->n_sel, base_pos, ctx->cfg.n, mask, position_ids, ctx->ws.status);
+    launch_after(ot::mask_kernel, dim3(B), dim3(ot::kSmallThreads), 0, static_cast<cudaStream_t>(stream),
+                 tree->parent, tree->depth, tree->n_sel, base_pos, ctx->cfg.n, mask, position_ids, ctx->ws.status);
     ctx->launches++;
     return check_launch();
 }
@@ -688,8 +703,8 @@ int opt_tree_verify(opt_tree_ctx* ctx, const opt_tree_out* tree, const void* tar
         B < 1 || B > ctx->cfg.max_batch)
         return OPT_TREE_ERR_INVALID_ARG;
     const ot::Params p = make_params(ctx, target, 0.0f);
-    ot::verify_kernel<<<dim3(ctx->cfg.n + 1, B), ot::kSmallThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        ctx->ws, p, static_cast<const uint16_t*>(target), root_token, *tree, accept_len, accept_tokens, accept_nodes, next_root);
+    launch_after(ot::verify_kernel, dim3(ctx->cfg.n + 1, B), dim3(ot::kSmallThreads), 0, static_cast<cudaStream_t>(stream),
+                 ctx->ws, p, static_cast<const uint16_t*>(target), root_token, *tree, accept_len, accept_tokens, accept_nodes, next_root);
     ctx->launches++;
     return check_launch();
 }

@@ -217,6 +217,7 @@ __device__ void finisher_role(CtaSmem& s, Sink& sink, int fidx, int V, int k, bo
 template <class Source, class Sink>
 __device__ __forceinline__ void run_pipeline(CtaSmem& s, Source& src, Sink& sink, int V, int k, bool aligned, int* status) {
     pipeline_init(s);
+    grid_dependency_wait();                                // shared memory is set up; global memory from here on
     const int warp = threadIdx.x >> 5;
     if (warp < kConsumerWarps) { consumer_role(s, warp, V, status); return; }
     const int helper = warp - kConsumerWarps;
