@@ -14,7 +14,11 @@
 namespace ot {
 
 constexpr int kRowMul = 31;                 // row of (token t, depth d) = (t*31 + d) mod H
-constexpr int kSmallThreads = 256;          // block size of the mask / verify / init kernels
+constexpr int kSmallThreads = 256;          // block size of the mask / init kernels
+// Verify: one CTA per target row.  With 128 threads sixteen CTAs fit an SM, so the n + 1 rows of 32
+// sequences (c4: 2080 CTAs) are all resident at once instead of in two uneven waves; a thread keeps
+// eight 16-byte loads in flight.
+constexpr int kVerifyThreads = 128;
 
 __device__ __forceinline__ int row_of(int token, int depth, int H) {
     return (int)(((long long)token * kRowMul + depth) % H);
@@ -435,7 +439,7 @@ __device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
 }
 
 struct VerifySmem {
-    unsigned long long red_u64[kSmallThreads / 32];
+    unsigned long long red_u64[kVerifyThreads / 32];
     int flag;
     int hit;
 };
@@ -443,7 +447,7 @@ struct VerifySmem {
 // Greedy verification.  CTA (j, b): j = 0 takes the target row after the root, j >= 1 the row after
 // kept node j-1; each finds the row's argmax (lowest token on ties).  The last CTA of a sequence
 // then walks the tree: accept the child that carries the target's token, until none does.
-__global__ void __launch_bounds__(kSmallThreads)
+__global__ void __launch_bounds__(kVerifyThreads)
 verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const int32_t* __restrict__ root_token,
               opt_tree_out tree, int32_t* accept_len, int32_t* accept_tokens, int32_t* accept_nodes, int32_t* next_root) {
     __shared__ VerifySmem s;
@@ -464,23 +468,19 @@ verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const 
         const int nv = p.V >> 3;
         float best = -INFINITY;
         int best_v = -1;
-        int v = tid;
-        for (; v + 3 * kSmallThreads < nv; v += 4 * kSmallThreads) {
-            uint4 q[4];
+#pragma unroll 1
+        for (int v0 = tid; v0 < nv; v0 += 8 * kVerifyThreads) {
+            uint4 q[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) q[u] = ld_nc_v4(vec + v + u * kSmallThreads);
+            for (int u = 0; u < 8; ++u)
+                q[u] = v0 + u * kVerifyThreads < nv ? ld_nc_v4(vec + v0 + u * kVerifyThreads)
+                                                    : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < 8; ++u) {
                 const uint32_t m2 = max_bf16x2(max_bf16x2(q[u].x, q[u].y), max_bf16x2(q[u].z, q[u].w));
                 const float f = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
-                if (f > best || best_v < 0) { best = f; best_v = v + u * kSmallThreads; }
+                if (v0 + u * kVerifyThreads < nv && (f > best || best_v < 0)) { best = f; best_v = v0 + u * kVerifyThreads; }
             }
-        }
-        for (; v < nv; v += kSmallThreads) {
-            const uint4 q = ld_nc_v4(vec + v);
-            const uint32_t m2 = max_bf16x2(max_bf16x2(q.x, q.y), max_bf16x2(q.z, q.w));
-            const float f = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
-            if (f > best || best_v < 0) { best = f; best_v = v; }
         }
         if (best_v >= 0) {
             const uint4 q = vec[best_v];
@@ -492,7 +492,7 @@ verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const 
             }
         }
     } else {
-        for (int v = tid; v < p.V; v += kSmallThreads) {
+        for (int v = tid; v < p.V; v += kVerifyThreads) {
             const unsigned long long key = cand_key(__ldg(row + v), (uint32_t)v);
             best_key = key > best_key ? key : best_key;
         }
@@ -502,7 +502,7 @@ verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const 
     __syncthreads();
     int32_t* g = w.g + (size_t)b * (p.n + 1);
     if (tid == 0) {
-        for (int q = 1; q < kSmallThreads / 32; ++q) best_key = s.red_u64[q] > best_key ? s.red_u64[q] : best_key;
+        for (int q = 1; q < kVerifyThreads / 32; ++q) best_key = s.red_u64[q] > best_key ? s.red_u64[q] : best_key;
         g[j] = (int32_t)cand_token(best_key);
         __threadfence();
         s.flag = (atomicAdd(&w.vdone[b], 1) == ns);
@@ -514,8 +514,8 @@ verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const 
     // acceptance walk (block-wide child search; children of one node carry distinct tokens)
     int32_t* at = accept_tokens + (size_t)b * (p.max_depth + 1);
     int32_t* an = accept_nodes + (size_t)b * p.max_depth;
-    for (int i = tid; i <= p.max_depth; i += kSmallThreads) at[i] = -1;
-    for (int i = tid; i < p.max_depth; i += kSmallThreads) an[i] = -1;
+    for (int i = tid; i <= p.max_depth; i += kVerifyThreads) at[i] = -1;
+    for (int i = tid; i < p.max_depth; i += kVerifyThreads) an[i] = -1;
     __syncthreads();
     int cur = -1, A = 0;
     for (int step = 0; step <= p.max_depth; ++step) {
@@ -524,7 +524,7 @@ verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const 
         ++A;
         __syncthreads();
         if (A > p.max_depth) break;
-        for (int i = tid; i < ns; i += kSmallThreads)
+        for (int i = tid; i < ns; i += kVerifyThreads)
             if (par[i] == cur && tok[i] == y) s.hit = i;
         __syncthreads();
         const int hit = s.hit;
@@ -703,7 +703,7 @@ int opt_tree_verify(opt_tree_ctx* ctx, const opt_tree_out* tree, const void* tar
         B < 1 || B > ctx->cfg.max_batch)
         return OPT_TREE_ERR_INVALID_ARG;
     const ot::Params p = make_params(ctx, target, 0.0f);
-    launch_after(ot::verify_kernel, dim3(ctx->cfg.n + 1, B), dim3(ot::kSmallThreads), 0, static_cast<cudaStream_t>(stream),
+    launch_after(ot::verify_kernel, dim3(ctx->cfg.n + 1, B), dim3(ot::kVerifyThreads), 0, static_cast<cudaStream_t>(stream),
                  ctx->ws, p, static_cast<const uint16_t*>(target), root_token, *tree, accept_len, accept_tokens, accept_nodes, next_root);
     ctx->launches++;
     return check_launch();
@@ -839,7 +839,7 @@ extern "C" int opt_tree_verify_static(const opt_tree_config* cfg, const opt_tree
     p.V = cfg->V; p.H = cfg->H; p.n = cfg->n; p.k = cfg->k; p.kk = cfg->k < cfg->V ? cfg->k : cfg->V;
     p.max_depth = cfg->max_depth; p.Dcap = cfg->max_depth < cfg->n ? cfg->max_depth : cfg->n;
     p.aligned = ((reinterpret_cast<uintptr_t>(target) & 15u) == 0 && (cfg->V % 8) == 0) ? 1 : 0;
-    ot::verify_kernel<<<dim3(cfg->n + 1, B), ot::kSmallThreads, 0, st>>>(
+    ot::verify_kernel<<<dim3(cfg->n + 1, B), ot::kVerifyThreads, 0, st>>>(
         ws, p, static_cast<const uint16_t*>(target), root_token, *tree, accept_len, accept_tokens, accept_nodes, next_root);
     if (cudaGetLastError() != cudaSuccess) return OPT_TREE_ERR_CUDA;
     if (device_status && cudaMemcpyAsync(device_status, ws.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
