@@ -171,6 +171,23 @@ def mask_of(parent, depth, n_sel: int, n: int, base_pos: int = 0):
     return mask, pos
 
 
+def dense_mask_of(parent, n_sel: int, n: int) -> np.ndarray:
+    """[n+1][n+1] uint8: who attends to whom inside one step (position 0 = root, i+1 = node i)."""
+    parent = np.ascontiguousarray(parent, np.int32)
+    dense = np.zeros((n + 1, n + 1), np.uint8)
+    lib().ot_dense_mask(_p(parent, C.c_int32), C.c_int32(n_sel), C.c_int32(n), _p(dense, C.c_uint8))
+    return dense
+
+
+def kv_keep_of(accept_nodes, accept_len: int, max_depth: int):
+    """(gather [max_depth+1] int32, kept): the step positions whose keys and values stay cached, in path order."""
+    an = np.ascontiguousarray(accept_nodes, np.int32)
+    gather = np.empty(max_depth + 1, np.int32)
+    lib().ot_kv_keep.restype = C.c_int32
+    kept = lib().ot_kv_keep(_p(an, C.c_int32), C.c_int32(accept_len), C.c_int32(max_depth), _p(gather, C.c_int32))
+    return gather, int(kept)
+
+
 def row_softmax_topk(row_bf16: np.ndarray, k: int):
     """(tokens, probs, m, S) of one bf16 row."""
     row = np.ascontiguousarray(row_bf16, np.uint16)

@@ -413,6 +413,40 @@ void ot_mask(const int32_t *parent, const int32_t *depth, int32_t n_sel, int32_t
 }
 
 /* ------------------------------------------------------------------------- */
+/* Bookkeeping around the target forward of Algorithm 2 (the step after the  */
+/* hot path).  The paper says only that the tree attention mask is computed  */
+/* and that both models keep key and value caches (Section 3, after          */
+/* Algorithm 2); the formats below are this build's reading:                 */
+/*  - the target sees n+1 tokens per step: position 0 is the root (the last  */
+/*    accepted token), position i+1 is packed node i;                        */
+/*  - dense mask [n+1][n+1]: entry (r, c) is 1 iff token r may attend to     */
+/*    token c inside the step: c == r, or r is a kept node and c is the root */
+/*    or one of r's ancestors.  Unused positions attend to themselves only;  */
+/*  - after Verify the keys and values of the root and of the A-1 matched    */
+/*    nodes stay in the cache, in path order: gather[0] = 0, gather[j] =     */
+/*    1 + accept_nodes[j-1]; the rest of gather is -1; A entries are kept    */
+/*    (the A-th accepted token is the next step's root and has no entry yet).*/
+/* ------------------------------------------------------------------------- */
+void ot_dense_mask(const int32_t *parent, int32_t n_sel, int32_t n, uint8_t *dense)
+{
+    const int32_t S = n + 1;
+    memset(dense, 0, (size_t)S * S);
+    for (int32_t r = 0; r < S; ++r) dense[(size_t)r * S + r] = 1;
+    for (int32_t i = 0; i < n_sel; ++i) {
+        dense[(size_t)(i + 1) * S + 0] = 1;
+        for (int32_t a = parent[i]; a >= 0; a = parent[a]) dense[(size_t)(i + 1) * S + (a + 1)] = 1;
+    }
+}
+
+int32_t ot_kv_keep(const int32_t *accept_nodes, int32_t accept_len, int32_t max_depth, int32_t *gather)
+{
+    for (int32_t j = 0; j <= max_depth; ++j) gather[j] = -1;
+    gather[0] = 0;
+    for (int32_t j = 1; j < accept_len; ++j) gather[j] = 1 + accept_nodes[j - 1];
+    return accept_len;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Greedy verification: the target's most probable next token after the root */
 /* and after every tree node; accept the longest root branch that follows    */
 /* them, plus the next token after the last hit.                             */
