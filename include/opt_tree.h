@@ -154,6 +154,26 @@ int opt_tree_verify_static(const opt_tree_config *cfg, const opt_tree_out *tree,
 int opt_tree_row_softmax_topk(opt_tree_ctx *ctx, const void *logits_bf16, const int32_t *rows,
                               int32_t nrows, int32_t *tok_out, double *prob_out, void *stream);
 
+/* Bookkeeping after verification (Algorithm 2: the mask that M(T_opt, mask) consumes, in dense
+ * form; Section 3, last paragraph: both models keep key and value caches, so after Verify only
+ * the accepted tokens' entries stay).  The paper fixes neither format; this library's are:
+ * the target sees n+1 tokens per step, position 0 the root (the last accepted token), position
+ * i+1 packed node i.
+ *   mask        (dev) [B][n][W]      bitmask written by opt_tree_mask
+ *   accept_len, accept_nodes (dev)   as written by opt_tree_verify
+ *   dense_mask  (dev) [B][n+1][n+1] uint8: 1 iff the row's token may attend to the column's token
+ *               inside the step (itself; for a kept node also the root and its ancestors); unused
+ *               positions attend to themselves only
+ *   kv_gather   (dev) [B][max_depth+1] int32: step positions whose keys and values stay cached, in
+ *               path order (0 = root, then 1 + accept_nodes[j]); -1 beyond kv_keep
+ *   kv_keep     (dev) [B] int32: entries kept = accept_len (the last accepted token is the next
+ *               step's root and has no entry yet)
+ * Enqueues one kernel on `stream`; returns OPT_TREE_ERR_INVALID_ARG for null pointers or B out of
+ * range.  Reads and writes only the caller's arrays and the context's status word. */
+int opt_tree_post_verify(opt_tree_ctx *ctx, const opt_tree_out *tree, const uint64_t *mask,
+                         const int32_t *accept_len, const int32_t *accept_nodes, int32_t B,
+                         uint8_t *dense_mask, int32_t *kv_gather, int32_t *kv_keep, void *stream);
+
 /* One whole decoding step (build, mask, verify) with HOST buffers: copies root_token and
  * base_pos to the device, runs the three stages, copies every output back and synchronises the
  * stream before returning.  The logit tables stay on the device (they stand in for the models).

@@ -19,7 +19,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -
 
 EXPORTS = ["opt_tree_workspace_bytes", "opt_tree_create", "opt_tree_destroy", "opt_tree_build", "opt_tree_mask",
            "opt_tree_verify", "opt_tree_row_softmax_topk", "opt_tree_step_host", "opt_tree_last_device_status",
-           "opt_tree_launch_count", "opt_tree_strerror", "opt_tree_verify_static"]
+           "opt_tree_launch_count", "opt_tree_strerror", "opt_tree_verify_static", "opt_tree_post_verify"]
 
 
 class Config(C.Structure):
@@ -65,6 +65,8 @@ def lib():
         L.opt_tree_launch_count.argtypes = [C.c_void_p]
         L.opt_tree_verify_static.argtypes = [C.POINTER(Config), C.POINTER(Out), C.c_void_p, C.c_void_p, C.c_int32,
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.opt_tree_post_verify.argtypes = [C.c_void_p, C.POINTER(Out), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.opt_tree_strerror.restype = C.c_char_p
         L.opt_tree_strerror.argtypes = [C.c_int]
         _lib = L
@@ -171,6 +173,18 @@ class OptTree:
         cs = tree.c_struct()
         _check(lib().opt_tree_verify(self._ctx, C.byref(cs), _ptr(target), _ptr(root_token), B,
                                      _ptr(out[0]), _ptr(out[1]), _ptr(out[2]), _ptr(out[3]), _stream()), "opt_tree_verify")
+        return out
+
+    def post_verify(self, tree: Tree, mask: torch.Tensor, accept_len: torch.Tensor, accept_nodes: torch.Tensor, out=None):
+        """Dense (n+1)x(n+1) attention mask and the cache keep list of the accepted path."""
+        B, n, D = tree.token.shape[0], self.cfg.n, self.cfg.max_depth
+        if out is None:
+            out = (torch.empty((B, n + 1, n + 1), dtype=torch.uint8, device=self.device),
+                   torch.empty((B, D + 1), dtype=torch.int32, device=self.device),
+                   torch.empty(B, dtype=torch.int32, device=self.device))
+        cs = tree.c_struct()
+        _check(lib().opt_tree_post_verify(self._ctx, C.byref(cs), _ptr(mask), _ptr(accept_len), _ptr(accept_nodes), B,
+                                          _ptr(out[0]), _ptr(out[1]), _ptr(out[2]), _stream()), "opt_tree_post_verify")
         return out
 
     def row_softmax_topk(self, logits: torch.Tensor, rows: torch.Tensor):

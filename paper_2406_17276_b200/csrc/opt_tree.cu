@@ -431,6 +431,43 @@ mask_kernel(const int32_t* __restrict__ parent, const int32_t* __restrict__ dept
     position_ids[(size_t)b * n + i] = pos;
 }
 
+// After verification: the bitmask expanded to the dense (n+1) x (n+1) form, position 0 being the
+// root, and the step positions whose keys and values stay in the caches (the root and the matched
+// nodes, in path order).  One CTA per sequence.
+__global__ void __launch_bounds__(kSmallThreads)
+post_verify_kernel(const int32_t* __restrict__ n_sel, const uint64_t* __restrict__ mask, const int32_t* __restrict__ accept_len,
+                   const int32_t* __restrict__ accept_nodes, int n, int max_depth, uint8_t* dense, int32_t* kv_gather,
+                   int32_t* kv_keep, int* status) {
+    grid_dependency_wait();
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int S = n + 1, W = (n + 63) >> 6;
+    const int ns = n_sel[b];
+    const uint64_t* mb = mask + (size_t)b * n * W;
+    uint8_t* db = dense + (size_t)b * S * S;
+    for (int idx = tid; idx < S * S; idx += kSmallThreads) {
+        const int r = idx / S, c = idx - r * S;
+        bool on = r == c;
+        if (r >= 1 && r - 1 < ns) {
+            if (c == 0) on = true;
+            else on = (mb[(size_t)(r - 1) * W + ((c - 1) >> 6)] >> ((c - 1) & 63)) & 1ull;
+        }
+        db[idx] = on ? 1 : 0;
+    }
+    int A = accept_len[b];
+    if (A < 1 || A > max_depth + 1) { set_status(status, kErrInternal); A = 1; }
+    for (int j = tid; j <= max_depth; j += kSmallThreads) {
+        int g = -1;
+        if (j == 0) g = 0;
+        else if (j < A) {
+            const int node = accept_nodes[(size_t)b * max_depth + j - 1];
+            if (node < 0 || node >= ns) set_status(status, kErrInternal);
+            else g = 1 + node;
+        }
+        kv_gather[(size_t)b * (max_depth + 1) + j] = g;
+    }
+    if (tid == 0) kv_keep[b] = A;
+}
+
 __device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -705,6 +742,19 @@ int opt_tree_verify(opt_tree_ctx* ctx, const opt_tree_out* tree, const void* tar
     const ot::Params p = make_params(ctx, target, 0.0f);
     launch_after(ot::verify_kernel, dim3(ctx->cfg.n + 1, B), dim3(ot::kVerifyThreads), 0, static_cast<cudaStream_t>(stream),
                  ctx->ws, p, static_cast<const uint16_t*>(target), root_token, *tree, accept_len, accept_tokens, accept_nodes, next_root);
+    ctx->launches++;
+    return check_launch();
+}
+
+int opt_tree_post_verify(opt_tree_ctx* ctx, const opt_tree_out* tree, const uint64_t* mask, const int32_t* accept_len,
+                         const int32_t* accept_nodes, int32_t B, uint8_t* dense_mask, int32_t* kv_gather, int32_t* kv_keep,
+                         void* stream) {
+    if (!ctx || bad_tree(tree) || !mask || !accept_len || !accept_nodes || !dense_mask || !kv_gather || !kv_keep || B < 1 ||
+        B > ctx->cfg.max_batch)
+        return OPT_TREE_ERR_INVALID_ARG;
+    launch_after(ot::post_verify_kernel, dim3(B), dim3(ot::kSmallThreads), 0, static_cast<cudaStream_t>(stream),
+                 tree->n_sel, mask, accept_len, accept_nodes, ctx->cfg.n, ctx->cfg.max_depth, dense_mask, kv_gather, kv_keep,
+                 ctx->ws.status);
     ctx->launches++;
     return check_launch();
 }
