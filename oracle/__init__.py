@@ -120,6 +120,27 @@ def table_step(draft: np.ndarray, target: np.ndarray | None, root_token: np.ndar
     return r
 
 
+def table_build_rows(draft: np.ndarray, root_token: np.ndarray, n: int, k: int, max_depth: int, delta: float, prune: bool):
+    """Trees of a batch on the table model, full or pruned (only layer nodes still among the n largest
+    are drafted from), and the draft rows each sequence read.  Returns (StepResult-like dict, rows)."""
+    H, V = draft.shape
+    root_token = np.ascontiguousarray(root_token, dtype=np.int32)
+    B = root_token.shape[0]
+    out = dict(token=np.empty((B, n), np.int32), parent=np.empty((B, n), np.int32), depth=np.empty((B, n), np.int32),
+               phat=np.empty((B, n), np.float64), n_sel=np.empty(B, np.int32), depth_reached=np.empty(B, np.int32),
+               expected_len=np.empty(B, np.float64), esub_trace=np.zeros((B, max_depth), np.float64))
+    rows = np.zeros(B, np.int64)
+    rc = lib().ot_table_build_rows(
+        _p(draft, C.c_uint16), C.c_int32(H), C.c_int32(V), _p(root_token, C.c_int32), C.c_int32(B),
+        C.c_int32(n), C.c_int32(k), C.c_int32(max_depth), C.c_double(delta), C.c_int32(1 if prune else 0),
+        _p(out["token"], C.c_int32), _p(out["parent"], C.c_int32), _p(out["depth"], C.c_int32), _p(out["phat"], C.c_double),
+        _p(out["n_sel"], C.c_int32), _p(out["depth_reached"], C.c_int32), _p(out["expected_len"], C.c_double),
+        _p(out["esub_trace"], C.c_double), _p(rows, C.c_int64))
+    if rc != 0:
+        raise ValueError("oracle: bad arguments")
+    return out, rows
+
+
 def build_cb(logits_of, root_token: int, V: int, n: int, k: int, max_depth: int, delta: float,
              force_depth: int = 0):
     """Build one tree from a Python model: logits_of(root_token, path_tuple) -> sequence of V floats."""

@@ -265,11 +265,17 @@ static double rel_gap(double kept, double dropped)
  *   stop_margin                  smallest |gain - delta| over the threshold tests evaluated
  * Returns 0, or -1 on bad arguments.
  */
-int ot_build(const ot_model *model, ot_memo *memo, int32_t root_token,
+/* prune != 0: the variant that drafts, of every new layer, only the nodes that are among the n
+ * largest of T at that moment.  By Theorem 1 a node's descendants have smaller path values than the
+ * node, so the descendants of a node outside the n largest can never be among the n largest later:
+ * T_opt, E_sub after every layer and the loop test come out the same, with fewer draft rows read
+ * (rows_read counts them).  Once no node of the newest layer is among the n largest, further layers
+ * change nothing; the loop then only replays its test, as the full version would. */
+static int build_impl(const ot_model *model, ot_memo *memo, int32_t root_token,
              int32_t V, int32_t n, int32_t k, int32_t max_depth, double delta, int32_t force_depth,
              int32_t *token, int32_t *parent, int32_t *depth, double *phat,
              int32_t *n_sel, int32_t *depth_reached, double *expected_len,
-             double *esub_trace, double *min_gap, double *stop_margin)
+             double *esub_trace, double *min_gap, double *stop_margin, int32_t prune, int64_t *rows_read)
 {
     if (V < 1 || n < 1 || k < 1 || max_depth < 1) return -1;
     int32_t D = max_depth < n ? max_depth : n;       /* Algorithm 1 loop: depth of tree < n */
@@ -284,17 +290,20 @@ int ot_build(const ot_model *model, ot_memo *memo, int32_t root_token,
     int32_t *path = (int32_t *)malloc((size_t)(D + 1) * sizeof(int32_t));
 
     double E = 0.0, Esub = 0.0, gapmin = INFINITY, margin = INFINITY;
-    int32_t frontier_begin = -1, frontier_end = -1;   /* [begin,end) in T; -1 = the root */
+    int32_t *front = (int32_t *)malloc((size_t)n * sizeof(int32_t));   /* nodes of T to draft from; -1 = the root */
+    int32_t nfront = 1;
+    front[0] = -1;
     int32_t d = 0, nR = 0;
+    int64_t rows = 0;
     for (int32_t i = 0; i < max_depth; ++i) esub_trace[i] = 0.0;
 
     for (;;) {
         d += 1;
-        /* Draft step: next-token distribution of every node in the last layer. */
+        /* Draft step: next-token distribution of every node to draft from. */
         int32_t ncand = 0;
-        int32_t nfront = frontier_begin < 0 ? 1 : frontier_end - frontier_begin;
+        rows += nfront;
         for (int32_t s = 0; s < nfront; ++s) {
-            int32_t f = frontier_begin < 0 ? -1 : frontier_begin + s;
+            int32_t f = front[s];
             double fphat = 1.0;                       /* root: factor 1 */
             int32_t fdepth = 0;
             if (f >= 0) {
@@ -321,9 +330,8 @@ int ot_build(const ot_model *model, ot_memo *memo, int32_t root_token,
             if (g < gapmin) gapmin = g;
         }
         qsort(cands, (size_t)nl, sizeof *cands, cmp_cidx_asc);
-        frontier_begin = nT;
+        int32_t layer_begin = nT;
         for (int32_t i = 0; i < nl; ++i) T[nT++] = cands[i];
-        frontier_end = nT;
 
         /* E_sub(T, n): the n largest path values of T (closure proof after Algorithm 1). */
         for (int32_t i = 0; i < nT; ++i) {
@@ -338,6 +346,16 @@ int ot_build(const ot_model *model, ot_memo *memo, int32_t root_token,
             if (g < gapmin) gapmin = g;
         }
         esub_trace[d - 1] = Esub;
+
+        /* Who is drafted from next: the whole new layer, or (prune) its members among the n largest. */
+        nfront = 0;
+        for (int32_t i = layer_begin; i < nT; ++i) {
+            int32_t in_top = 0;
+            if (prune) {
+                for (int32_t q = 0; q < nR; ++q) if (R[q].id == i) { in_top = 1; break; }
+            }
+            if (!prune || in_top) front[nfront++] = i;
+        }
 
         /* Loop test of Algorithm 1. */
         if (d >= D) break;
@@ -387,8 +405,39 @@ int ot_build(const ot_model *model, ot_memo *memo, int32_t root_token,
     *expected_len = EA;
     if (min_gap) *min_gap = gapmin;
     if (stop_margin) *stop_margin = margin;
+    if (rows_read) *rows_read = rows;
 
-    free(C); free(canon_of); free(T); free(cands); free(R); free(scratch); free(ctok); free(cp); free(path);
+    free(C); free(canon_of); free(T); free(cands); free(R); free(scratch); free(ctok); free(cp); free(path); free(front);
+    return 0;
+}
+
+int ot_build(const ot_model *model, ot_memo *memo, int32_t root_token,
+             int32_t V, int32_t n, int32_t k, int32_t max_depth, double delta, int32_t force_depth,
+             int32_t *token, int32_t *parent, int32_t *depth, double *phat,
+             int32_t *n_sel, int32_t *depth_reached, double *expected_len,
+             double *esub_trace, double *min_gap, double *stop_margin)
+{
+    return build_impl(model, memo, root_token, V, n, k, max_depth, delta, force_depth, token, parent, depth, phat,
+                      n_sel, depth_reached, expected_len, esub_trace, min_gap, stop_margin, 0, NULL);
+}
+
+/* The pruned variant over the table model for a batch (tree outputs and the number of draft rows
+ * each sequence read; with prune == 0 the full version, for comparison of the row counts). */
+int ot_table_build_rows(const uint16_t *draft, int32_t H, int32_t V, const int32_t *root_token, int32_t batch,
+                        int32_t n, int32_t k, int32_t max_depth, double delta, int32_t prune,
+                        int32_t *token, int32_t *parent, int32_t *depth, double *phat,
+                        int32_t *n_sel, int32_t *depth_reached, double *expected_len, double *esub_trace,
+                        int64_t *rows_read)
+{
+    ot_table_model dm = { draft, H, V };
+    ot_model dmodel = { ot_table_logits, ot_table_key, &dm };
+    for (int32_t b = 0; b < batch; ++b) {
+        int rc = build_impl(&dmodel, NULL, root_token[b], V, n, k, max_depth, delta, 0,
+                            token + (size_t)b * n, parent + (size_t)b * n, depth + (size_t)b * n, phat + (size_t)b * n,
+                            n_sel + b, depth_reached + b, expected_len + b, esub_trace + (size_t)b * max_depth,
+                            NULL, NULL, prune, rows_read + b);
+        if (rc) return rc;
+    }
     return 0;
 }
 
