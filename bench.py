@@ -231,6 +231,21 @@ def run_cuda(args):
     if ot.device_status() != 0:
         raise SystemExit("bench.py: device status after post_verify")
 
+    # ---- the pruned draft (same trees from fewer rows): timed on its own, with its own byte count ----
+    rows_read = torch.empty(B, dtype=torch.int32, device="cuda")
+    for _ in range(5):
+        ot.build_pruned(d_ld, roots0, delta, tree, rows_read)
+    q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    q0.record()
+    for _ in range(50):
+        ot.build_pruned(d_ld, roots0, delta, tree, rows_read)
+    q1.record(); torch.cuda.synchronize()
+    pruned_ms = q0.elapsed_time(q1) / 50
+    pruned_rows = int(rows_read.sum().item())
+    if ot.device_status() != 0:
+        raise SystemExit("bench.py: device status after build_pruned")
+
     peak, peak_kind = _peaks()
     achieved = algo_bytes / (build_ms * 1e-3) / 1e9
     line = {
@@ -246,6 +261,9 @@ def run_cuda(args):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches),
+        "pruned_build": {"ms_per_build": pruned_ms, "trees_per_s": B / (pruned_ms * 1e-3), "rows_read": pruned_rows,
+                         "rows_of_full_build": int(rows_total), "gbs_of_rows_read": 2.0 * w.V * pruned_rows / (pruned_ms * 1e-3) / 1e9,
+                         "note": "opt_tree_build_pruned alone on the first step's roots: the same trees, only rows that can still matter; not the benchmark's metric"},
         "post_verify": {"us_per_call": post_verify_us, "bytes_written": int(sum(t.numel() * t.element_size() for t in pv_out)),
                         "note": "opt_tree_post_verify alone, 100 back-to-back calls; not part of the timed step"},
         "roofline": {"bound": "hbm", "kernel": "build_kernel (opt_tree_build: init_build_kernel + one persistent build_kernel)",

@@ -154,6 +154,18 @@ int opt_tree_verify_static(const opt_tree_config *cfg, const opt_tree_out *tree,
 int opt_tree_row_softmax_topk(opt_tree_ctx *ctx, const void *logits_bf16, const int32_t *rows,
                               int32_t nrows, int32_t *tok_out, double *prob_out, void *stream);
 
+/* opt_tree_build with frontier pruning: of every new layer only the nodes that are among the n
+ * largest of T at that moment are drafted from (their rows of the draft table are the only ones
+ * read).  By Theorem 1 a node's descendants have smaller path values than the node, so what is
+ * left out can never reach the n largest: the outputs (tree, E(A), E_sub trace, depth_reached)
+ * are those of opt_tree_build, for fewer rows.  Algorithm 1 as printed drafts from the whole last
+ * layer; this variant is the one Section 3 has in mind when it notes that the input of a
+ * drafting step is at most n tokens.
+ *   rows_read (dev) [B] int32 or NULL: draft rows each sequence read (the root's included)
+ * Arguments, ownership and errors otherwise as opt_tree_build. */
+int opt_tree_build_pruned(opt_tree_ctx *ctx, const void *draft_logits_bf16, const int32_t *root_token,
+                          int32_t B, float delta, const opt_tree_out *out, int32_t *rows_read, void *stream);
+
 /* Bookkeeping after verification (Algorithm 2: the mask that M(T_opt, mask) consumes, in dense
  * form; Section 3, last paragraph: both models keep key and value caches, so after Verify only
  * the accepted tokens' entries stay).  The paper fixes neither format; this library's are:

@@ -19,7 +19,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -
 
 EXPORTS = ["opt_tree_workspace_bytes", "opt_tree_create", "opt_tree_destroy", "opt_tree_build", "opt_tree_mask",
            "opt_tree_verify", "opt_tree_row_softmax_topk", "opt_tree_step_host", "opt_tree_last_device_status",
-           "opt_tree_launch_count", "opt_tree_strerror", "opt_tree_verify_static", "opt_tree_post_verify"]
+           "opt_tree_launch_count", "opt_tree_strerror", "opt_tree_verify_static", "opt_tree_post_verify", "opt_tree_build_pruned"]
 
 
 class Config(C.Structure):
@@ -65,6 +65,8 @@ def lib():
         L.opt_tree_launch_count.argtypes = [C.c_void_p]
         L.opt_tree_verify_static.argtypes = [C.POINTER(Config), C.POINTER(Out), C.c_void_p, C.c_void_p, C.c_int32,
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.opt_tree_build_pruned.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_float, C.POINTER(Out), C.c_void_p,
+                                            C.c_void_p]
         L.opt_tree_post_verify.argtypes = [C.c_void_p, C.POINTER(Out), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.opt_tree_strerror.restype = C.c_char_p
@@ -151,6 +153,18 @@ class OptTree:
         _check(lib().opt_tree_build(self._ctx, _ptr(draft), _ptr(root_token), B, C.c_float(delta), C.byref(cs), _stream()),
                "opt_tree_build")
         return out
+
+    def build_pruned(self, draft: torch.Tensor, root_token: torch.Tensor, delta: float, out: Tree | None = None,
+                     rows_read: torch.Tensor | None = None):
+        """opt_tree_build_pruned: the same trees from fewer draft rows; returns (tree, rows_read [B] int32)."""
+        B = root_token.shape[0]
+        out = out or self.alloc_tree(B)
+        if rows_read is None:
+            rows_read = torch.empty(B, dtype=torch.int32, device=self.device)
+        cs = out.c_struct()
+        _check(lib().opt_tree_build_pruned(self._ctx, _ptr(draft), _ptr(root_token), B, C.c_float(delta), C.byref(cs),
+                                           _ptr(rows_read), _stream()), "opt_tree_build_pruned")
+        return out, rows_read
 
     def mask(self, tree: Tree, base_pos: torch.Tensor | None = None, mask: torch.Tensor | None = None,
              position_ids: torch.Tensor | None = None):

@@ -37,6 +37,7 @@ struct Workspace {
     int32_t* R;            // [B][2][n]
     double* E_prev;        // [B]
     int32_t* st;           // [B][8]
+    int32_t* fmap;         // [B][n]   pruned draft: layer slot behind each frontier row
     // row mailboxes of the build: one per CTA, filled by the layer warps, never wrapped within a build.
     // The rows of a build are numbered by one running count (q_ctl[kQCursor]): row g goes to CTA
     // g % grid, entry g / grid of its mailbox.
@@ -93,6 +94,7 @@ static size_t carve(const opt_tree_config& c, int grid, char* base, Workspace* w
     OT_TAKE(R, int32_t, B * 2 * n)
     OT_TAKE(E_prev, double, B)
     OT_TAKE(st, int32_t, B * 8)
+    OT_TAKE(fmap, int32_t, B * n)
     OT_TAKE(mb_items, unsigned long long, mailbox_capacity(c, grid) * grid)
     OT_TAKE(mb_phat, unsigned long long, mailbox_capacity(c, grid) * grid)
     OT_TAKE(q_ctl, int32_t, 8)
@@ -123,6 +125,7 @@ struct Params {            // by-value kernel parameters
     float delta;
     int aligned;
     int mcap, grid, cstride;
+    int prune;             // draft only from layer nodes that are still among the n largest
 };
 
 __device__ __forceinline__ SeqWork seq_work(const Workspace& w, const Params& p, int b) {
@@ -135,6 +138,7 @@ __device__ __forceinline__ SeqWork seq_work(const Workspace& w, const Params& p,
     s.R = w.R + (size_t)b * 2 * p.n;
     s.E_prev = w.E_prev + b;
     s.st = w.st + (size_t)b * 8;
+    s.fmap = w.fmap + (size_t)b * p.n;
     return s;
 }
 __device__ __forceinline__ TreeOut tree_out(const opt_tree_out& o, const Params& p, int b) {
@@ -190,7 +194,8 @@ __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restri
     }
     if (i < p.B) {
         int32_t* st = w.st + (size_t)i * 8;
-        st[kStDone] = 0; st[kStNR] = 0;
+        st[kStDone] = 0; st[kStNR] = 0; st[kStRows] = 0;
+        w.fmap[(size_t)i * p.n] = 0;                                      // the root row stands for "slot 0"
         w.E_prev[i] = 0.0;
     }
     if (i == 0) { w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; w.q_ctl[kQCursor] = p.B; }   // the roots are rows 0 .. B-1
@@ -246,16 +251,21 @@ struct BuildSink {
         if ((threadIdx.x & 31) == 0) g0 = atomicAdd(reinterpret_cast<unsigned int*>(&w.q_ctl[kQCursor]), (unsigned)nl);
         return g0;
     }
-    __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl, unsigned g0) {
+    // pick != null (pruned draft): only the layer slots pick[0..nl) are sent out, as frontier rows 0..nl;
+    // the map from frontier row to layer slot is left in fmap for the next selection.
+    __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl, unsigned g0, const int* pick = nullptr,
+                                  int32_t* fmap = nullptr) {
         const int lane = threadIdx.x & 31;
         g0 = __shfl_sync(0xFFFFFFFFu, g0, 0);
         for (int i = lane; i < nl; i += 32) {
-            int token = ls.ltok[i];
+            const int slot = pick ? pick[i] : i;
+            if (fmap) fmap[i] = slot;
+            int token = ls.ltok[slot];
             if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
             const unsigned g = g0 + (unsigned)i, c = g % (unsigned)p.grid, e = g / (unsigned)p.grid;
             if (e < (unsigned)p.mcap) {
                 const size_t pos = (size_t)c * p.mcap + e;
-                st_relaxed_u64(&w.mb_phat[pos], (1ull << 63) | (ls.lkeys[i] - 1ull));
+                st_relaxed_u64(&w.mb_phat[pos], (1ull << 63) | (ls.lkeys[slot] - 1ull));
                 st_relaxed_u64(&w.mb_items[pos], item_encode(b, d + 1, i, row_of(token, d, p.H)));
             } else {
                 set_status(w.status, kErrInternal);
@@ -311,7 +321,7 @@ struct BuildSink {
                     const int nvalid = fsize * p.kk, nl = nvalid < p.n ? nvalid : p.n;
                     // Without a threshold the loop test only looks at the depth: the next layer's rows
                     // can go out before the running top-n is brought up to date.
-                    const bool early = d < p.Dcap && p.delta == -INFINITY;
+                    const bool early = d < p.Dcap && p.delta == -INFINITY && !p.prune;
                     stage_layer_candidates(ls, sw, fsize, p.k);
                     unsigned g0 = 0;
                     if (early) g0 = reserve_layer(nl);        // the rows' numbers, while the candidates load
@@ -322,6 +332,7 @@ struct BuildSink {
                             j.kind = 1; j.d = d; j.fsize = fsize; j.n = p.n; j.k = p.k; j.kk = p.kk;
                             j.cand_phat = sw.cand_phat; j.cand_tok = sw.cand_tok;
                             j.T_tok = sw.T_tok; j.T_par = sw.T_par; j.T_phat = sw.T_phat;
+                            j.fmap = p.prune ? sw.fmap : nullptr;
                         }
                         if (small) cp_async_wait_all();       // the staged candidates are in shared memory
                         __syncwarp();
@@ -331,13 +342,39 @@ struct BuildSink {
                         else select_layer_team_big(ls, j, lane, w.status);
                     }
                     if (early) publish_layer(ls, b, d, nl, g0);
-                    const bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta,
-                                                          w.status);
-                    if (more && !early) {
+                    int nR = 0;
+                    double esub = 0.0;
+                    bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta,
+                                                    w.status, nR, esub);
+                    int sent = nl;                             // rows of the next layer
+                    if (more && p.prune) {
+                        // The new layer's nodes among the n largest are the tail of the ascending list rsel
+                        // (their gids are the largest); only they are drafted from.
+                        const int gid0 = (d - 1) * p.n;
+                        int mine = 0;
+                        for (int i = lane; i < nR; i += 32) mine += ls.rsel[i] >= gid0 ? 1 : 0;
+                        sent = __reduce_add_sync(0xFFFFFFFFu, mine);
+                        for (int i = lane; i < sent; i += 32) ls.gids[i] = ls.rsel[nR - sent + i] - gid0;
+                        __syncwarp();
+                        if (sent > 0) {
+                            publish_layer(ls, b, d, sent, reserve_layer(sent), ls.gids, sw.fmap);
+                        } else {
+                            // Nothing left to draft from: further layers change neither T_opt nor E_sub.  The loop
+                            // of Algorithm 1 would go on testing a gain of zero: to the depth limit if the
+                            // threshold is negative, else for one more layer.
+                            const int d_end = p.delta < 0.0f ? p.Dcap : d + 1;
+                            const TreeOut to = tree_out(out, p, b);
+                            if (to.esub_trace) for (int i = d + lane; i < d_end; i += 32) to.esub_trace[i] = esub;
+                            __syncwarp();
+                            pack_tree_warp(ls, sw, to, d_end, nR, p.n, p.max_depth, esub, w.status);
+                            more = false;
+                        }
+                    } else if (more && !early) {
                         publish_layer(ls, b, d, nl, reserve_layer(nl));
                     }
-                    if (more) { cur_d[q] = d + 1; cur_f[q] = nl; cur_tot[q] += nl; }
-                    else {
+                    if (more) { cur_d[q] = d + 1; cur_f[q] = sent; cur_tot[q] += sent; }
+                    if (lane == 0) sw.st[kStRows] = cur_tot[q];
+                    if (!more) {
                         cur_d[q] = 0; --live;
                         __threadfence();
                         if (lane == 0 && atomicAdd(&w.q_ctl[kQFinished], 1) == p.B - 1) st_release_s32(&w.q_ctl[kQDone], 1);
@@ -615,6 +652,7 @@ ot::Params make_params(const opt_tree_ctx* ctx, const void* table, float delta) 
     p.Dcap = c.max_depth < c.n ? c.max_depth : c.n;
     p.max_depth = c.max_depth;
     p.B = 0;
+    p.prune = 0;
     p.mcap = ctx->mcap;
     p.grid = ctx->grid;
     p.cstride = (int)ot::cand_stride(c.n, c.k);
@@ -710,19 +748,35 @@ int opt_tree_destroy(opt_tree_ctx* ctx) {
     return e == cudaSuccess ? OPT_TREE_OK : OPT_TREE_ERR_CUDA;
 }
 
-int opt_tree_build(opt_tree_ctx* ctx, const void* draft, const int32_t* root_token, int32_t B, float delta,
-                   const opt_tree_out* out, void* stream) {
+static int build_common(opt_tree_ctx* ctx, const void* draft, const int32_t* root_token, int32_t B, float delta,
+                        const opt_tree_out* out, int prune, int32_t* rows_read, void* stream) {
     if (!ctx || !draft || !root_token || bad_tree(out) || B < 1 || delta != delta) return OPT_TREE_ERR_INVALID_ARG;
     if (B > ctx->cfg.max_batch) return OPT_TREE_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     ot::Params p = make_params(ctx, draft, delta);
     p.B = B;
+    p.prune = prune;
     const long long init_threads = (long long)ctx->grid * ctx->mcap > B ? (long long)ctx->grid * ctx->mcap : B;
     launch_after(ot::init_build_kernel, dim3((unsigned)((init_threads + 255) / 256)), dim3(256), 0, st, ctx->ws, p, root_token);
     launch_after(ot::build_kernel, dim3(ctx->grid), dim3(ot::kThreads), sizeof(ot::CtaSmem), st,
                  ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
     ctx->launches += 2;
-    return check_launch();
+    int rc = check_launch();
+    if (rc == OPT_TREE_OK && rows_read &&
+        cudaMemcpy2DAsync(rows_read, sizeof(int32_t), ctx->ws.st + ot::kStRows, 8 * sizeof(int32_t), sizeof(int32_t), (size_t)B,
+                          cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        rc = OPT_TREE_ERR_CUDA;
+    return rc;
+}
+
+int opt_tree_build(opt_tree_ctx* ctx, const void* draft, const int32_t* root_token, int32_t B, float delta,
+                   const opt_tree_out* out, void* stream) {
+    return build_common(ctx, draft, root_token, B, delta, out, 0, nullptr, stream);
+}
+
+int opt_tree_build_pruned(opt_tree_ctx* ctx, const void* draft, const int32_t* root_token, int32_t B, float delta,
+                          const opt_tree_out* out, int32_t* rows_read, void* stream) {
+    return build_common(ctx, draft, root_token, B, delta, out, 1, rows_read, stream);
 }
 
 int opt_tree_mask(opt_tree_ctx* ctx, const opt_tree_out* tree, int32_t B, const int32_t* base_pos, uint64_t* mask,

@@ -74,6 +74,7 @@ struct alignas(16) FinScratch {    // private to one finisher warp (hist is clea
 struct LayerJob {                  // what the layer warp hands its assistants (kind 0: leave)
     int kind, d, fsize, n, k, kk;
     double* cand_phat; int32_t* cand_tok; int32_t* T_tok; int32_t* T_par; double* T_phat;
+    const int32_t* fmap;           // pruned draft: layer slot of the node behind each frontier row (null: the identity)
 };
 
 struct alignas(16) LayerScratch {  // private to the layer team of a CTA

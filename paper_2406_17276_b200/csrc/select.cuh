@@ -117,9 +117,10 @@ struct SeqWork {
     double* T_phat;        // [D*n]
     int32_t* R;            // [2][n]   running top-n as gids in ascending order, double-buffered by layer parity
     double* E_prev;        // [1]      E of Algorithm 1
-    int32_t* st;           // [8]      1: rows finished since the build began, 2: |R|
+    int32_t* st;           // [8]      1: rows finished since the build began, 2: |R|, 3: rows sent out in all
+    int32_t* fmap;         // [n]      pruned draft: layer slot of the node behind each frontier row
 };
-enum { kStDone = 1, kStNR = 2 };
+enum { kStDone = 1, kStNR = 2, kStRows = 3 };
 
 struct TreeOut {           // mirrors opt_tree_out, pointers offset to the sequence
     int32_t *token, *parent, *depth;
@@ -329,7 +330,7 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
             const int tok = t32 == ~0u ? -1 : (int)(t32 & 0x7FFFFFFFu);
             j.T_tok[gid0 + pos] = tok;
             s.ltok[pos] = tok;
-            j.T_par[gid0 + pos] = i / j.k;
+            j.T_par[gid0 + pos] = j.fmap ? __ldcg(&j.fmap[i / j.k]) : i / j.k;
             j.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
             s.lkeys[pos] = key;
             ++pos;
@@ -410,7 +411,7 @@ __device__ __noinline__ int select_layer_team_big(LayerScratch& s, const LayerJo
                 const int tok = t32 == ~0u ? -1 : (int)(t32 & 0x7FFFFFFFu);
                 j.T_tok[gid0 + pos] = tok;
                 s.ltok[pos] = tok;
-                j.T_par[gid0 + pos] = i / j.k;
+                j.T_par[gid0 + pos] = j.fmap ? __ldcg(&j.fmap[i / j.k]) : i / j.k;
                 j.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
                 s.lkeys[pos] = key;
                 ++pos;
@@ -463,7 +464,7 @@ __device__ __noinline__ void pack_tree_warp(LayerScratch& s, const SeqWork& w, c
 // finished.  All layers of a sequence are handled by the same warp, in order.  Returns true if the
 // sequence continues with layer d+1, false if it is finished (outputs written).
 __device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
-                                    int max_depth, float delta, int* status) {
+                                    int max_depth, float delta, int* status, int& nR_out, double& esub_out) {
     const int lane = threadIdx.x & 31;
     int* hist = s.hist;
     const int gid0 = (d - 1) * n;
@@ -508,6 +509,7 @@ __device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork&
         *w.E_prev = esub;
     }
     __syncwarp();
+    nR_out = nR; esub_out = esub;
     if (more) return true;
     pack_tree_warp(s, w, out, d, nR, n, max_depth, esub, status);
     return false;
