@@ -225,6 +225,9 @@ struct BuildSource {
 // counter.  Layer warp: the layer warp of CTA c owns sequences c, c + gridDim.x, ...; it watches
 // their row counters, and when a layer is complete does the layer selection, publishes the next
 // layer's rows, brings the running top-n up to date and applies the loop test of Algorithm 1.
+// kPrune: the pruned draft (opt_tree_build_pruned); a compile-time choice so that the ordinary build
+// carries none of its code.
+template <bool kPrune>
 struct BuildSink {
     Workspace w; Params p; opt_tree_out out;
     __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch&) {
@@ -288,8 +291,8 @@ struct BuildSink {
             team_sync();
             const LayerJob j = ls.job;
             if (j.kind == 0) return;
-            if (j.fsize * j.k <= 1024) select_layer_team(ls, j, tt, w.status);
-            else select_layer_team_big(ls, j, tt, w.status);
+            if (j.fsize * j.k <= 1024) select_layer_team<kPrune>(ls, j, tt, w.status);
+            else select_layer_team_big<kPrune>(ls, j, tt, w.status);
         }
     }
     __device__ void layer_follow(LayerScratch& ls) {
@@ -321,7 +324,7 @@ struct BuildSink {
                     const int nvalid = fsize * p.kk, nl = nvalid < p.n ? nvalid : p.n;
                     // Without a threshold the loop test only looks at the depth: the next layer's rows
                     // can go out before the running top-n is brought up to date.
-                    const bool early = d < p.Dcap && p.delta == -INFINITY && !p.prune;
+                    const bool early = !kPrune && d < p.Dcap && p.delta == -INFINITY;
                     stage_layer_candidates(ls, sw, fsize, p.k);
                     unsigned g0 = 0;
                     if (early) g0 = reserve_layer(nl);        // the rows' numbers, while the candidates load
@@ -332,25 +335,25 @@ struct BuildSink {
                             j.kind = 1; j.d = d; j.fsize = fsize; j.n = p.n; j.k = p.k; j.kk = p.kk;
                             j.cand_phat = sw.cand_phat; j.cand_tok = sw.cand_tok;
                             j.T_tok = sw.T_tok; j.T_par = sw.T_par; j.T_phat = sw.T_phat;
-                            j.fmap = p.prune ? sw.fmap : nullptr;
+                            j.fmap = kPrune ? sw.fmap : nullptr;
                         }
                         if (small) cp_async_wait_all();       // the staged candidates are in shared memory
                         __syncwarp();
                         team_sync();                          // ... and, with the job, visible to the assistants
                         const LayerJob j = ls.job;
-                        if (small) select_layer_team(ls, j, lane, w.status);
-                        else select_layer_team_big(ls, j, lane, w.status);
+                        if (small) select_layer_team<kPrune>(ls, j, lane, w.status);
+                        else select_layer_team_big<kPrune>(ls, j, lane, w.status);
                     }
                     if (early) publish_layer(ls, b, d, nl, g0);
-                    int nR = 0;
-                    double esub = 0.0;
                     bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta,
-                                                    w.status, nR, esub);
+                                                    w.status);
                     int sent = nl;                             // rows of the next layer
-                    if (more && p.prune) {
+                    if (kPrune && more) {
                         // The new layer's nodes among the n largest are the tail of the ascending list rsel
                         // (their gids are the largest); only they are drafted from.
                         const int gid0 = (d - 1) * p.n;
+                        const int nR = ls.last_nR;
+                        const double esub = ls.last_esub;
                         int mine = 0;
                         for (int i = lane; i < nR; i += 32) mine += ls.rsel[i] >= gid0 ? 1 : 0;
                         sent = __reduce_add_sync(0xFFFFFFFFu, mine);
@@ -373,7 +376,7 @@ struct BuildSink {
                         publish_layer(ls, b, d, nl, reserve_layer(nl));
                     }
                     if (more) { cur_d[q] = d + 1; cur_f[q] = sent; cur_tot[q] += sent; }
-                    if (lane == 0) sw.st[kStRows] = cur_tot[q];
+                    if (kPrune && lane == 0) sw.st[kStRows] = cur_tot[q];
                     if (!more) {
                         cur_d[q] = 0; --live;
                         __threadfence();
@@ -393,12 +396,13 @@ struct BuildSink {
 
 // Algorithm 1 for a whole batch in one launch: persistent CTAs take rows from their mailboxes; layers
 // of different sequences overlap freely because sequences never exchange data.
+template <bool kPrune>
 __global__ void __launch_bounds__(kThreads)
 build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, opt_tree_out out) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
     BuildSource src{w, p, draft};
-    BuildSink sink{w, p, out};
+    BuildSink<kPrune> sink{w, p, out};
     run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, w.status);
 }
 
@@ -686,9 +690,10 @@ extern "C" {
 static int persistent_grid() {
     int dev = 0, per_sm = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
-    if (cudaFuncSetAttribute(ot::build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
+    if (cudaFuncSetAttribute(ot::build_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::build_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
         cudaFuncSetAttribute(ot::row_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ot::build_kernel, ot::kThreads, sizeof(ot::CtaSmem)) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ot::build_kernel<true>, ot::kThreads, sizeof(ot::CtaSmem)) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
         cudaGetLastError();
         return 0;
@@ -758,8 +763,12 @@ static int build_common(opt_tree_ctx* ctx, const void* draft, const int32_t* roo
     p.prune = prune;
     const long long init_threads = (long long)ctx->grid * ctx->mcap > B ? (long long)ctx->grid * ctx->mcap : B;
     launch_after(ot::init_build_kernel, dim3((unsigned)((init_threads + 255) / 256)), dim3(256), 0, st, ctx->ws, p, root_token);
-    launch_after(ot::build_kernel, dim3(ctx->grid), dim3(ot::kThreads), sizeof(ot::CtaSmem), st,
-                 ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
+    if (prune)
+        launch_after(ot::build_kernel<true>, dim3(ctx->grid), dim3(ot::kThreads), sizeof(ot::CtaSmem), st,
+                     ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
+    else
+        launch_after(ot::build_kernel<false>, dim3(ctx->grid), dim3(ot::kThreads), sizeof(ot::CtaSmem), st,
+                     ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
     ctx->launches += 2;
     int rc = check_launch();
     if (rc == OPT_TREE_OK && rows_read &&

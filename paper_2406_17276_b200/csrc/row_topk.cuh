@@ -90,6 +90,8 @@ struct alignas(16) LayerScratch {  // private to the layer team of a CTA
     unsigned long long red_or[kTeamWarps], red_and[kTeamWarps];
     int scan_a[kTeamWarps], scan_b[kTeamWarps];
     LayerJob job;
+    double last_esub;                          // E_sub and |R| of the last update of the running top-n
+    int last_nR;
 };
 
 static_assert(sizeof(RowSlot) % 16 == 0, "slots must keep 16-byte alignment in an array");

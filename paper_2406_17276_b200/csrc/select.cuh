@@ -267,6 +267,7 @@ __device__ int team_radix_select(LayerScratch& s, const unsigned long long* gw, 
 // The team's part of a layer selection (N = fsize * k <= 1024; the candidates were staged into s
 // by the layer warp).  On return (after a last barrier) the new layer's nodes are in T and its
 // tokens and keys in s.ltok / s.lkeys.  Returns nl.
+template <bool kPrune>
 __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j, int tt, int* status) {
     const int lane = threadIdx.x & 31, tw = tt >> 5;
     const int N = j.fsize * j.k;
@@ -330,7 +331,7 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
             const int tok = t32 == ~0u ? -1 : (int)(t32 & 0x7FFFFFFFu);
             j.T_tok[gid0 + pos] = tok;
             s.ltok[pos] = tok;
-            j.T_par[gid0 + pos] = j.fmap ? __ldcg(&j.fmap[i / j.k]) : i / j.k;
+            j.T_par[gid0 + pos] = kPrune ? __ldcg(&j.fmap[i / j.k]) : i / j.k;
             j.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
             s.lkeys[pos] = key;
             ++pos;
@@ -344,6 +345,7 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
 // The team's selection for layers with more candidates than the shared-memory staging holds
 // (1024 < N <= n*k): the same steps, but every sweep reads the candidate words from global memory
 // (they sit in L2), a thread's loads eight at a time.  The candidate arrays are cleared at the end.
+template <bool kPrune>
 __device__ __noinline__ int select_layer_team_big(LayerScratch& s, const LayerJob& j, int tt, int* status) {
     const int lane = threadIdx.x & 31, tw = tt >> 5;
     const int N = j.fsize * j.k;
@@ -411,7 +413,7 @@ __device__ __noinline__ int select_layer_team_big(LayerScratch& s, const LayerJo
                 const int tok = t32 == ~0u ? -1 : (int)(t32 & 0x7FFFFFFFu);
                 j.T_tok[gid0 + pos] = tok;
                 s.ltok[pos] = tok;
-                j.T_par[gid0 + pos] = j.fmap ? __ldcg(&j.fmap[i / j.k]) : i / j.k;
+                j.T_par[gid0 + pos] = kPrune ? __ldcg(&j.fmap[i / j.k]) : i / j.k;
                 j.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
                 s.lkeys[pos] = key;
                 ++pos;
@@ -464,7 +466,7 @@ __device__ __noinline__ void pack_tree_warp(LayerScratch& s, const SeqWork& w, c
 // finished.  All layers of a sequence are handled by the same warp, in order.  Returns true if the
 // sequence continues with layer d+1, false if it is finished (outputs written).
 __device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
-                                    int max_depth, float delta, int* status, int& nR_out, double& esub_out) {
+                                    int max_depth, float delta, int* status) {
     const int lane = threadIdx.x & 31;
     int* hist = s.hist;
     const int gid0 = (d - 1) * n;
@@ -509,7 +511,8 @@ __device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork&
         *w.E_prev = esub;
     }
     __syncwarp();
-    nR_out = nR; esub_out = esub;
+    if (lane == 0) { s.last_nR = nR; s.last_esub = esub; }
+    __syncwarp();
     if (more) return true;
     pack_tree_warp(s, w, out, d, nR, n, max_depth, esub, status);
     return false;
