@@ -164,6 +164,10 @@ __device__ __forceinline__ unsigned long long item_encode(int b, int d, int slot
            ((unsigned long long)slot << 22) | (unsigned long long)row;
 }
 
+// An entry that was handed out but is not needed after all (the pruned draft reserves a layer's entries
+// before it knows how many rows the layer will have): fetchers drop such a ticket.
+constexpr unsigned long long kItemVoid = 1ull << 38;
+
 __device__ __forceinline__ unsigned long long phat_word(double p) {
     return (1ull << 63) | (unsigned long long)__double_as_longlong(p);
 }
@@ -211,6 +215,7 @@ struct BuildSource {
     __device__ int poll(long long idx, RowDesc& d, bool check_done) {
         const unsigned long long item = ld_relaxed_u64(&w.mb_items[idx]), ph = ld_relaxed_u64(&w.mb_phat[idx]);
         if (!((item & ph) >> 63)) return check_done && ld_acquire_s32(&w.q_ctl[kQDone]) ? -1 : 0;
+        if (item & kItemVoid) return 2;
         d.b = (int)((item >> 48) & 0x7FFFu); d.d = (int)((item >> 39) & 0x1FFu);
         d.slot = (int)((item >> 22) & 0xFFu); d.fsize = 0;
         d.pphat = __longlong_as_double((long long)(ph & 0x7FFFFFFFFFFFFFFFull));
@@ -276,6 +281,86 @@ struct BuildSink {
         }
         __syncwarp();
     }
+    // Entries g0+from .. g0+to of a reservation are not needed.
+    __device__ void void_entries(unsigned g0, int from, int to) {
+        const int lane = threadIdx.x & 31;
+        g0 = __shfl_sync(0xFFFFFFFFu, g0, 0);
+        for (int i = from + lane; i < to; i += 32) {
+            const unsigned g = g0 + (unsigned)i, c = g % (unsigned)p.grid, e = g / (unsigned)p.grid;
+            if (e < (unsigned)p.mcap) {
+                const size_t pos = (size_t)c * p.mcap + e;
+                st_relaxed_u64(&w.mb_phat[pos], 1ull << 63);
+                st_relaxed_u64(&w.mb_items[pos], (1ull << 63) | kItemVoid);
+            } else {
+                set_status(w.status, kErrInternal);
+            }
+        }
+        __syncwarp();
+    }
+    // Pruned draft, a whole layer job with one selection (see select_running_team).  Returns the number
+    // of rows of the next layer, or -1 if the sequence is finished.
+    __device__ int merged_layer_job(LayerScratch& ls, const SeqWork& sw, int b, int d, int fsize, int nR_old, int off) {
+        const int lane = threadIdx.x & 31;
+        const int nvalid = fsize * p.kk, reserve = nvalid < p.n ? nvalid : p.n;
+        stage_layer_candidates(ls, sw, fsize, p.k, off);
+        const unsigned g0 = d < p.Dcap ? reserve_layer(reserve) : 0u;      // entries for the next layer, before its size is known
+        // the old top-n: still in the scratch if this warp's last job was this sequence's previous layer
+        const int32_t* Rold = sw.R + ((d - 1) & 1) * p.n;
+        const bool cached = ls.cache_b == b && ls.cache_d == d - 1;
+        for (int i = lane; i < nR_old; i += 32) {
+            int gid;
+            unsigned long long key;
+            if (cached) { gid = ls.rsel[i]; key = phat_key(ls.vals[i]); }
+            else { gid = __ldcg(&Rold[i]); key = phat_key(__ldcg(&sw.T_phat[gid])); }
+            ls.gids[i] = gid;
+            ls.keys[i] = key;
+        }
+        if (lane == 0) {
+            LayerJob& j = ls.job;
+            j.kind = 2; j.d = d; j.fsize = fsize; j.n = p.n; j.k = p.k; j.kk = p.kk;
+            j.cand_phat = sw.cand_phat; j.cand_tok = sw.cand_tok;
+            j.T_tok = sw.T_tok; j.T_par = sw.T_par; j.T_phat = sw.T_phat;
+            j.fmap = sw.fmap; j.nR_old = nR_old; j.off = off; j.Rnew = sw.R + (d & 1) * p.n;
+        }
+        cp_async_wait_all();
+        __syncwarp();
+        team_sync();
+        const LayerJob j = ls.job;
+        const int nR = select_running_team(ls, j, lane, w.status);
+        int kept_old = 0;
+#pragma unroll
+        for (int q = 0; q < kTeamWarps; ++q) kept_old += ls.scan_c[q];
+        const int cnt = nR - kept_old;                      // new members = the rows of the next layer
+        double part = 0.0;
+        for (int i = lane; i < nR; i += 32) part += ls.vals[i];
+        const double esub = warp_sum(part);
+        const double eprev = d == 1 ? 0.0 : __ldcg(sw.E_prev);
+        bool more = d < p.Dcap && (esub - eprev > (double)p.delta);
+        const TreeOut to = tree_out(out, p, b);
+        if (lane == 0) {
+            if (to.esub_trace) to.esub_trace[d - 1] = esub;
+            sw.st[kStNR] = nR;
+            *sw.E_prev = esub;
+            ls.cache_b = b; ls.cache_d = d;
+        }
+        __syncwarp();
+        if (more && cnt > 0) {
+            for (int i = lane; i < cnt; i += 32) ls.gids[i] = i;       // members are sent out in slot order
+            __syncwarp();
+            publish_layer(ls, b, d, cnt, g0, ls.gids, sw.fmap);
+            void_entries(g0, cnt, reserve);
+            return cnt;
+        }
+        if (d < p.Dcap) void_entries(g0, 0, reserve);
+        int d_end = d;
+        if (more) {                                         // nothing left to draft from: the loop would go on testing a gain of zero
+            d_end = p.delta < 0.0f ? p.Dcap : d + 1;
+            if (to.esub_trace) for (int i = d + lane; i < d_end; i += 32) to.esub_trace[i] = esub;
+            __syncwarp();
+        }
+        pack_tree_warp(ls, sw, to, d_end, nR, p.n, p.max_depth, esub, w.status);
+        return -1;
+    }
     // The layer warp follows its sequences (layer_follow); whenever a layer is complete it hands the
     // selection to the whole team: the job goes into shared memory, the team barrier starts it.  The
     // assistants wait at that barrier in between and leave when they find a job of kind 0.
@@ -291,7 +376,8 @@ struct BuildSink {
             team_sync();
             const LayerJob j = ls.job;
             if (j.kind == 0) return;
-            if (j.fsize * j.k <= 1024) select_layer_team<kPrune>(ls, j, tt, w.status);
+            if (kPrune && j.kind == 2) select_running_team(ls, j, tt, w.status);
+            else if (j.fsize * j.k <= 1024) select_layer_team<kPrune>(ls, j, tt, w.status);
             else select_layer_team_big<kPrune>(ls, j, tt, w.status);
         }
     }
@@ -324,6 +410,22 @@ struct BuildSink {
                     const int nvalid = fsize * p.kk, nl = nvalid < p.n ? nvalid : p.n;
                     // Without a threshold the loop test only looks at the depth: the next layer's rows
                     // can go out before the running top-n is brought up to date.
+                    if (kPrune) {
+                        const int nR_old = d == 1 ? 0 : __ldcg(&sw.st[kStNR]);
+                        const int off = (nR_old + 1) & ~1;
+                        if (off + fsize * p.k <= 1024) {
+                            const int sent = merged_layer_job(ls, sw, b, d, fsize, nR_old, off);
+                            if (sent > 0) { cur_d[q] = d + 1; cur_f[q] = sent; cur_tot[q] += sent; }
+                            if (lane == 0) sw.st[kStRows] = cur_tot[q];
+                            if (sent <= 0) {
+                                cur_d[q] = 0; --live;
+                                __threadfence();
+                                if (lane == 0 && atomicAdd(&w.q_ctl[kQFinished], 1) == p.B - 1) st_release_s32(&w.q_ctl[kQDone], 1);
+                            }
+                            __syncwarp();
+                            continue;
+                        }
+                    }
                     const bool early = !kPrune && d < p.Dcap && p.delta == -INFINITY;
                     stage_layer_candidates(ls, sw, fsize, p.k);
                     unsigned g0 = 0;
@@ -347,6 +449,7 @@ struct BuildSink {
                     if (early) publish_layer(ls, b, d, nl, g0);
                     bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta,
                                                     w.status);
+                    if (kPrune && lane == 0) { ls.cache_b = b; ls.cache_d = d; }     // rsel / vals now hold this top-n
                     int sent = nl;                             // rows of the next layer
                     if (kPrune && more) {
                         // The new layer's nodes among the n largest are the tail of the ascending list rsel

@@ -37,6 +37,7 @@ __device__ __forceinline__ void pipeline_init(CtaSmem& s) {
         mbar_fence_init();
     }
     for (int i = threadIdx.x; i < 3 * 256; i += kThreads) (&s.layer.thist[0][0])[i] = 0;
+    if (threadIdx.x == 0) { s.layer.cache_b = -1; s.layer.cache_d = -1; }
     __syncthreads();
 }
 
@@ -49,7 +50,7 @@ __device__ __forceinline__ void pipeline_init(CtaSmem& s) {
 // up a row that is ready.  Tickets are only taken while fewer than kDesc rows are between "ticket
 // taken" and "descriptor read by the consumers", which bounds what a CTA keeps from the others.
 //   Source::claim(i)          ticket for this CTA's i-th claim, or a negative value: no more work
-//   Source::poll(ticket, dsc) 1: descriptor filled, 0: not yet, -1: no more work
+//   Source::poll(ticket, dsc) 1: descriptor filled, 0: not yet, 2: the ticket turned out empty, -1: no more work
 // Once a Source has said "no more work" no ticket of this CTA can still turn into a row.
 constexpr int kFetchLanes = 4;
 template <class Source>
@@ -59,6 +60,7 @@ __device__ void fetcher_role(CtaSmem& s, Source& src, int* status) {
     bool holding = false;                 // this lane has a ticket
     long long ticket = 0;
     int claimed = 0, known = 0, consumed = 0;      // warp-uniform counts of this CTA's rows
+    int consumed_empty = 0;                        // tickets that turned out empty
     long long t0 = clock64();
     for (int turn = 0;; ++turn) {
         // rows whose descriptors the consumers have let go of
@@ -67,7 +69,7 @@ __device__ void fetcher_role(CtaSmem& s, Source& src, int* status) {
         const bool want = lane < kFetchLanes && !holding;
         const unsigned wm = __ballot_sync(0xFFFFFFFFu, want);
         const int my_claim = claimed + __popc(wm & below);
-        const bool take = want && my_claim - consumed < kDesc;
+        const bool take = want && my_claim - consumed_empty - consumed < kDesc;
         if (take) { ticket = src.claim(my_claim); holding = true; }
         claimed += __popc(__ballot_sync(0xFFFFFFFFu, take));
         // one poll per held ticket
@@ -75,6 +77,11 @@ __device__ void fetcher_role(CtaSmem& s, Source& src, int* status) {
         dsc.row = nullptr; dsc.pphat = 0.0; dsc.b = dsc.d = dsc.slot = dsc.fsize = 0; dsc.stop = 0;
         int got = 0;
         if (holding) got = ticket < 0 ? -1 : src.poll(ticket, dsc, (turn & 15) == 15);
+        {   // an entry that was handed out but not needed: the ticket is gone, and does not count as a row in hand
+            const bool empty = got == 2;
+            if (empty) { holding = false; got = 0; }
+            consumed_empty += __popc(__ballot_sync(0xFFFFFFFFu, empty));
+        }
         const unsigned rm = __ballot_sync(0xFFFFFFFFu, got > 0), em = __ballot_sync(0xFFFFFFFFu, got < 0);
         if (got > 0) {
             const int a = known + __popc(rm & below);

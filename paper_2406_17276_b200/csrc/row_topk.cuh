@@ -75,6 +75,9 @@ struct LayerJob {                  // what the layer warp hands its assistants (
     int kind, d, fsize, n, k, kk;
     double* cand_phat; int32_t* cand_tok; int32_t* T_tok; int32_t* T_par; double* T_phat;
     const int32_t* fmap;           // pruned draft: layer slot of the node behind each frontier row (null: the identity)
+    // kind 2 (pruned draft, one selection over the running top-n and the candidates together):
+    int nR_old, off;               // old top-n in keys[0..nR_old), candidates from keys[off] (off even, >= nR_old)
+    int32_t* Rnew;                 // the new top-n's gids, ascending
 };
 
 struct alignas(16) LayerScratch {  // private to the layer team of a CTA
@@ -92,6 +95,8 @@ struct alignas(16) LayerScratch {  // private to the layer team of a CTA
     LayerJob job;
     double last_esub;                          // E_sub and |R| of the last update of the running top-n
     int last_nR;
+    int scan_c[kTeamWarps];
+    int cache_b, cache_d;                      // rsel / vals hold the top-n of this sequence after this layer (-1: nothing)
 };
 
 static_assert(sizeof(RowSlot) % 16 == 0, "slots must keep 16-byte alignment in an array");

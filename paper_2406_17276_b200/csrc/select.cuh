@@ -133,14 +133,14 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
 // Starts the asynchronous copies of a layer's candidates (path values and tokens) into the layer
 // warp's scratch; the layer warp waits for them before it starts the team.  Separate so that other round trips (the
 // mailbox reservations) can be in flight at the same time.
-__device__ __forceinline__ void stage_layer_candidates(LayerScratch& s, const SeqWork& w, int fsize, int k) {
+__device__ __forceinline__ void stage_layer_candidates(LayerScratch& s, const SeqWork& w, int fsize, int k, int off = 0) {
     const int lane = threadIdx.x & 31;
     const int N = fsize * k;
-    if (N > 1024) return;
+    if (off + N > 1024) return;                            // (off is even: the copies keep their 16-byte alignment)
     const unsigned long long* gph = reinterpret_cast<const unsigned long long*>(w.cand_phat);
     const unsigned int* gtk = reinterpret_cast<const unsigned int*>(w.cand_tok);
     #pragma unroll 1
-    for (int i = lane * 2; i < N; i += 64) cp_async_16(&s.keys[i], &gph[i]);
+    for (int i = lane * 2; i < N; i += 64) cp_async_16(&s.keys[off + i], &gph[i]);
     #pragma unroll 1
     for (int i = lane * 4; i < N; i += 128) cp_async_16(&s.toks[i], &gtk[i]);
 }
@@ -340,6 +340,117 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
     if (total != nl) set_status(status, kErrInternal);
     team_sync();
     return nl;
+}
+
+// Pruned draft, both halves of a layer job in one selection: the new running top-n is the n largest
+// of the old one and the layer's candidates together (what a candidate outside them could add to T
+// can never matter, see opt_tree_build_pruned).  s.keys[0..nR_old) / s.gids[0..nR_old) hold the old
+// top-n (keys, gids ascending), s.keys[off..off+N) the staged candidate words (entries between are 0).
+// Array order is tie order (shallower first, then candidate index).  On return s.rsel / s.vals hold
+// the new top-n (gids ascending; also written to j.Rnew), its new members are T's nodes
+// gid0 .. gid0+cnt in candidate order with tokens and keys in s.ltok / s.lkeys, and s.scan_c sums
+// to the number of old members kept.  Returns |new top-n|.
+__device__ __noinline__ int select_running_team(LayerScratch& s, const LayerJob& j, int tt, int* status) {
+    const int lane = threadIdx.x & 31, tw = tt >> 5;
+    const int N = j.fsize * j.k, nRo = j.nR_old, off = j.off, M = off + N;
+    const int nvalid = j.fsize * j.kk;
+    const int need = nRo + nvalid < j.n ? nRo + nvalid : j.n;
+    const int gid0 = (j.d - 1) * j.n;
+    const unsigned long long* gph = reinterpret_cast<const unsigned long long*>(j.cand_phat);
+    const unsigned int* gtk = reinterpret_cast<const unsigned int*>(j.cand_tok);
+    unsigned long long ko = 0ull, ka = ~0ull;
+    #pragma unroll 1
+    for (int i = tt; i < M; i += kTeam) {
+        unsigned long long key;
+        if (i >= off) {
+            unsigned long long x = s.keys[i];
+            if (!(x >> 63)) x = poll_phat_word(&gph[i - off], status);
+            key = key_of_word(x);
+            s.keys[i] = key;
+            unsigned int t32 = (unsigned int)s.toks[i - off];
+            if (!(t32 >> 31)) { t32 = poll_tok_word(&gtk[i - off], status); s.toks[i - off] = (int)t32; }
+        } else {
+            key = i < nRo ? s.keys[i] : 0ull;
+            if (i >= nRo) s.keys[i] = 0ull;
+        }
+        if (key) { ko |= key; ka &= key; }
+    }
+    ko = warp_or_u64(ko); ka = warp_and_u64(ka);
+    if (lane == 0) { s.red_or[tw] = ko; s.red_and[tw] = ka; }
+    team_sync();
+    ko = 0ull; ka = ~0ull;
+#pragma unroll
+    for (int q = 0; q < kTeamWarps; ++q) { ko |= s.red_or[q]; ka &= s.red_and[q]; }
+    #pragma unroll 1
+    for (int i = tt * 2; i < N; i += 2 * kTeam) *reinterpret_cast<uint4*>(&j.cand_phat[i]) = make_uint4(0, 0, 0, 0);
+    #pragma unroll 1
+    for (int i = tt * 4; i < N; i += 4 * kTeam) *reinterpret_cast<uint4*>(&j.cand_tok[i]) = make_uint4(0, 0, 0, 0);
+    unsigned long long thr = 0ull;
+    int need_eq = 0, dirty = -1;
+    if (need < nRo + nvalid) dirty = team_radix_select<false>(s, nullptr, M, need, tt, ko, ka, thr, need_eq);
+    const int per = (M + kTeam - 1) / kTeam;
+    const int lo = min(tt * per, M), hi = min(lo + per, M);
+    int gt = 0, eq = 0;
+    #pragma unroll 1
+    for (int i = lo; i < hi; ++i) {
+        const unsigned long long key = s.keys[i];
+        gt += key > thr ? 1 : 0;
+        eq += (key == thr && key != 0ull) ? 1 : 0;
+    }
+    int total_eq, total;
+    int eq_take = 0;
+    if (need_eq > 0) {
+        const int eq_before = team_excl_scan(eq, s.scan_a, tw, total_eq);
+        eq_take = need_eq - eq_before;
+        eq_take = eq_take < 0 ? 0 : (eq_take > eq ? eq : eq_take);
+    }
+    // old members kept: counted per thread, summed over the team along with the scan below
+    int kept_mine = 0;
+    {
+        int e = eq_take;
+        #pragma unroll 1
+        for (int i = lo; i < hi && i < nRo; ++i) {
+            const unsigned long long key = s.keys[i];
+            bool take = key > thr;
+            if (key == thr && key != 0ull && e > 0) { take = true; --e; }
+            kept_mine += take ? 1 : 0;
+        }
+    }
+    kept_mine = __reduce_add_sync(0xFFFFFFFFu, kept_mine);
+    if (lane == 0) s.scan_c[tw] = kept_mine;
+    int pos = team_excl_scan(gt + eq_take, s.scan_b, tw, total);       // (its barrier also publishes scan_c)
+    if (dirty >= 0) { s.thist[dirty][tt] = 0; s.thist[dirty][tt + kTeam] = 0; }
+    int kept_old = 0;
+#pragma unroll
+    for (int q = 0; q < kTeamWarps; ++q) kept_old += s.scan_c[q];
+    #pragma unroll 1
+    for (int i = lo; i < hi; ++i) {
+        const unsigned long long key = s.keys[i];
+        bool take = key > thr;
+        if (key == thr && key != 0ull && eq_take > 0) { take = true; --eq_take; }
+        if (!take) continue;
+        int gid;
+        if (i < nRo) {
+            gid = s.gids[i];
+        } else {
+            const int c = i - off, slot = pos - kept_old;
+            const unsigned int t32 = (unsigned int)s.toks[c];
+            const int tok = t32 == ~0u ? -1 : (int)(t32 & 0x7FFFFFFFu);
+            gid = gid0 + slot;
+            j.T_tok[gid] = tok;
+            j.T_par[gid] = __ldcg(&j.fmap[c / j.k]);      // layer slot of the node behind the candidate's frontier row
+            j.T_phat[gid] = __longlong_as_double((long long)(key - 1ull));
+            s.ltok[slot] = tok;
+            s.lkeys[slot] = key;
+        }
+        s.rsel[pos] = gid;
+        s.vals[pos] = __longlong_as_double((long long)(key - 1ull));
+        j.Rnew[pos] = gid;
+        ++pos;
+    }
+    if (total != need) set_status(status, kErrInternal);
+    team_sync();
+    return need;
 }
 
 // The team's selection for layers with more candidates than the shared-memory staging holds
