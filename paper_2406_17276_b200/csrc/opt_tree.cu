@@ -206,7 +206,9 @@ __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restri
 }
 
 // Source of the tree build: the rows other CTAs' layer warps have put into this CTA's mailbox.
+template <bool kPrune>
 struct BuildSource {
+    static constexpr bool kHasEmpty = kPrune;              // only the pruned draft voids entries
     Workspace w; Params p;
     const uint16_t* draft;
     __device__ long long claim(int i) { return i < p.mcap ? (long long)blockIdx.x * p.mcap + i : -1; }
@@ -215,7 +217,7 @@ struct BuildSource {
     __device__ int poll(long long idx, RowDesc& d, bool check_done) {
         const unsigned long long item = ld_relaxed_u64(&w.mb_items[idx]), ph = ld_relaxed_u64(&w.mb_phat[idx]);
         if (!((item & ph) >> 63)) return check_done && ld_acquire_s32(&w.q_ctl[kQDone]) ? -1 : 0;
-        if (item & kItemVoid) return 2;
+        if (kPrune && (item & kItemVoid)) return 2;
         d.b = (int)((item >> 48) & 0x7FFFu); d.d = (int)((item >> 39) & 0x1FFu);
         d.slot = (int)((item >> 22) & 0xFFu); d.fsize = 0;
         d.pphat = __longlong_as_double((long long)(ph & 0x7FFFFFFFFFFFFFFFull));
@@ -504,13 +506,14 @@ __global__ void __launch_bounds__(kThreads)
 build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, opt_tree_out out) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
-    BuildSource src{w, p, draft};
+    BuildSource<kPrune> src{w, p, draft};
     BuildSink<kPrune> sink{w, p, out};
     run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, w.status);
 }
 
 // The row step alone over a list of rows (static round-robin over the CTAs).
 struct ListSource {
+    static constexpr bool kHasEmpty = false;
     const uint16_t* logits; const int32_t* rows; int nrows, V, H, first, stride; int* status;
     __device__ long long claim(int r) {
         const long long idx = (long long)first + (long long)r * stride;

@@ -77,7 +77,7 @@ __device__ void fetcher_role(CtaSmem& s, Source& src, int* status) {
         dsc.row = nullptr; dsc.pphat = 0.0; dsc.b = dsc.d = dsc.slot = dsc.fsize = 0; dsc.stop = 0;
         int got = 0;
         if (holding) got = ticket < 0 ? -1 : src.poll(ticket, dsc, (turn & 15) == 15);
-        {   // an entry that was handed out but not needed: the ticket is gone, and does not count as a row in hand
+        if (Source::kHasEmpty) {   // an entry that was handed out but not needed: the ticket is gone, and does not count as a row in hand
             const bool empty = got == 2;
             if (empty) { holding = false; got = 0; }
             consumed_empty += __popc(__ballot_sync(0xFFFFFFFFu, empty));
