@@ -166,6 +166,27 @@ int opt_tree_row_softmax_topk(opt_tree_ctx *ctx, const void *logits_bf16, const 
 int opt_tree_build_pruned(opt_tree_ctx *ctx, const void *draft_logits_bf16, const int32_t *root_token,
                           int32_t B, float delta, const opt_tree_out *out, int32_t *rows_read, void *stream);
 
+/* Layer-by-layer build, for a caller that runs a real draft model: Algorithm 1 with the draft step
+ * ("compute the next token distributions of the nodes in the last layer") left to the caller.
+ * opt_tree_layers_begin starts B trees; every opt_tree_layers_step takes the logits of the nodes
+ * that are to be expanded (first the root's, then each returned layer's), grows every tree by one
+ * layer exactly as opt_tree_build does (row softmax + top-k, Eq. 2, the n best candidates, E_sub,
+ * the loop test with `delta`) and returns the next layer; a tree whose growth stops is packed into
+ * `out` in that call.  The trees are those of opt_tree_build for the same logits.
+ *   frontier_logits (dev) bf16 [B][frontier_stride][V]: row f of sequence b belongs to node f of the
+ *                   layer returned by the previous step (the root for the first step); rows at or
+ *                   beyond a sequence's count are read but ignored.  1 <= frontier_stride <= n
+ *   out             as in opt_tree_build; written for a sequence when it stops
+ *   next_tokens     (dev) [B][n] int32  tokens of the new layer's nodes (to be expanded next)
+ *   next_parent     (dev) [B][n] int32  for each, the index of its parent in the previous layer
+ *   next_count      (dev) [B]   int32  nodes in the new layer; 0: this tree is finished
+ * One context builds one batch of trees at a time this way (the state lives in its workspace).
+ * Both calls only enqueue work on `stream`; errors as opt_tree_build. */
+int opt_tree_layers_begin(opt_tree_ctx *ctx, int32_t B, void *stream);
+int opt_tree_layers_step(opt_tree_ctx *ctx, const void *frontier_logits_bf16, int32_t frontier_stride, int32_t B,
+                         float delta, const opt_tree_out *out, int32_t *next_tokens, int32_t *next_parent,
+                         int32_t *next_count, void *stream);
+
 /* Bookkeeping after verification (Algorithm 2: the mask that M(T_opt, mask) consumes, in dense
  * form; Section 3, last paragraph: both models keep key and value caches, so after Verify only
  * the accepted tokens' entries stay).  The paper fixes neither format; this library's are:

@@ -19,7 +19,8 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -
 
 EXPORTS = ["opt_tree_workspace_bytes", "opt_tree_create", "opt_tree_destroy", "opt_tree_build", "opt_tree_mask",
            "opt_tree_verify", "opt_tree_row_softmax_topk", "opt_tree_step_host", "opt_tree_last_device_status",
-           "opt_tree_launch_count", "opt_tree_strerror", "opt_tree_verify_static", "opt_tree_post_verify", "opt_tree_build_pruned"]
+           "opt_tree_launch_count", "opt_tree_strerror", "opt_tree_verify_static", "opt_tree_post_verify", "opt_tree_build_pruned", "opt_tree_layers_begin",
+           "opt_tree_layers_step"]
 
 
 class Config(C.Structure):
@@ -67,6 +68,9 @@ def lib():
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.opt_tree_build_pruned.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_float, C.POINTER(Out), C.c_void_p,
                                             C.c_void_p]
+        L.opt_tree_layers_begin.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+        L.opt_tree_layers_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.POINTER(Out), C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_void_p]
         L.opt_tree_post_verify.argtypes = [C.c_void_p, C.POINTER(Out), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.opt_tree_strerror.restype = C.c_char_p
@@ -165,6 +169,21 @@ class OptTree:
         _check(lib().opt_tree_build_pruned(self._ctx, _ptr(draft), _ptr(root_token), B, C.c_float(delta), C.byref(cs),
                                            _ptr(rows_read), _stream()), "opt_tree_build_pruned")
         return out, rows_read
+
+    def layers_begin(self, B: int):
+        _check(lib().opt_tree_layers_begin(self._ctx, B, _stream()), "opt_tree_layers_begin")
+
+    def layers_step(self, frontier_logits: torch.Tensor, delta: float, tree: Tree, nxt=None):
+        """One layer of the layer-by-layer build; frontier_logits is [B][stride][V] bf16 bits on the device.
+        Returns (next_tokens [B][n], next_parent [B][n], next_count [B])."""
+        B, stride = frontier_logits.shape[0], frontier_logits.shape[1]
+        if nxt is None:
+            i32 = dict(dtype=torch.int32, device=self.device)
+            nxt = (torch.empty((B, self.cfg.n), **i32), torch.empty((B, self.cfg.n), **i32), torch.empty(B, **i32))
+        cs = tree.c_struct()
+        _check(lib().opt_tree_layers_step(self._ctx, _ptr(frontier_logits), stride, B, C.c_float(delta), C.byref(cs),
+                                          _ptr(nxt[0]), _ptr(nxt[1]), _ptr(nxt[2]), _stream()), "opt_tree_layers_step")
+        return nxt
 
     def mask(self, tree: Tree, base_pos: torch.Tensor | None = None, mask: torch.Tensor | None = None,
              position_ids: torch.Tensor | None = None):

@@ -38,6 +38,10 @@ struct Workspace {
     double* E_prev;        // [B]
     int32_t* st;           // [B][8]
     int32_t* fmap;         // [B][n]   pruned draft: layer slot behind each frontier row
+    // layer-by-layer build (logits handed in per layer)
+    double* front_phat;    // [B][n]   path values of the nodes whose logits come next
+    int32_t* rtok;         // [B*n][k] row results of the layer in hand
+    double* rprob;         // [B*n][k]
     // row mailboxes of the build: one per CTA, filled by the layer warps, never wrapped within a build.
     // The rows of a build are numbered by one running count (q_ctl[kQCursor]): row g goes to CTA
     // g % grid, entry g / grid of its mailbox.
@@ -95,6 +99,9 @@ static size_t carve(const opt_tree_config& c, int grid, char* base, Workspace* w
     OT_TAKE(E_prev, double, B)
     OT_TAKE(st, int32_t, B * 8)
     OT_TAKE(fmap, int32_t, B * n)
+    OT_TAKE(front_phat, double, B * n)
+    OT_TAKE(rtok, int32_t, B * n * (size_t)c.k)
+    OT_TAKE(rprob, double, B * n * (size_t)c.k)
     OT_TAKE(mb_items, unsigned long long, mailbox_capacity(c, grid) * grid)
     OT_TAKE(mb_phat, unsigned long long, mailbox_capacity(c, grid) * grid)
     OT_TAKE(q_ctl, int32_t, 8)
@@ -520,7 +527,7 @@ struct ListSource {
         return idx < nrows ? idx : -1;
     }
     __device__ int poll(long long idx, RowDesc& d, bool) {
-        int row = rows[idx];
+        int row = rows ? rows[idx] : (int)idx;             // no list: row idx of a dense buffer
         if (row < 0 || row >= H) { set_status(status, kErrInternal); row = 0; }
         d.row = logits + (size_t)row * V; d.slot = (int)idx; d.b = d.d = 0; d.fsize = 1;
         return 1;
@@ -546,6 +553,77 @@ row_topk_kernel(Params p, const uint16_t* __restrict__ logits, const int32_t* __
     ListSource src{logits, rows, nrows, p.V, p.H, (int)blockIdx.x, (int)gridDim.x, status};
     ListSink sink{tok_out, prob_out, p.k};
     run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, status);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Layer-by-layer build: the caller (a real draft model) hands in the logits of one layer's nodes at
+// a time.  Per layer one launch of the row kernel over the dense buffer and one of layer_step_kernel:
+// a CTA of kTeam threads per sequence forms the candidates (Eq. 2), selects the layer with the same
+// team selection as the persistent build, updates the running top-n / E_sub, applies the loop test
+// and hands back the next layer's tokens; a sequence that stops is packed on the spot.
+// ------------------------------------------------------------------------------------------------
+__global__ void layers_begin_kernel(Workspace w, Params p) {
+    grid_dependency_wait();
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= p.B) return;
+    int32_t* st = w.st + (size_t)b * 8;
+    st[kStDone] = 0; st[kStNR] = 0; st[kStRows] = 0; st[kStDepth] = 1; st[kStFsize] = 1;
+    w.E_prev[b] = 0.0;
+    w.front_phat[(size_t)b * p.n] = 1.0;                       // the root counts as factor 1
+    w.fmap[(size_t)b * p.n] = 0;
+}
+
+__global__ void __launch_bounds__(kTeam)
+layer_step_kernel(Workspace w, Params p, int fstride, opt_tree_out out, int32_t* next_tokens, int32_t* next_parent,
+                  int32_t* next_count) {
+    __shared__ LayerScratch ls;
+    grid_dependency_wait();
+    const int b = blockIdx.x, tt = threadIdx.x, lane = tt & 31;
+    for (int i = tt; i < 3 * 256; i += kTeam) (&ls.thist[0][0])[i] = 0;
+    const SeqWork sw = seq_work(w, p, b);
+    const int d = sw.st[kStDepth], fsize = sw.st[kStFsize];
+    if (d == 0) {                                            // this sequence stopped at an earlier layer
+        if (tt == 0) next_count[b] = 0;
+        return;
+    }
+    if (fsize < 1 || fsize > fstride || fsize > p.n) { if (tt == 0) { set_status(w.status, kErrInternal); next_count[b] = 0; } return; }
+    // candidates of the layer (Eq. 2), left the way the finishers of the persistent build leave them
+    const int N = fsize * p.k;
+    const double* fph = w.front_phat + (size_t)b * p.n;
+    for (int i = tt; i < N; i += kTeam) {
+        const int f = i / p.k, r = i - f * p.k;
+        const size_t src = ((size_t)b * fstride + f) * p.k + r;
+        const int tok = w.rtok[src];
+        const bool valid = r < p.kk && tok >= 0;
+        reinterpret_cast<unsigned long long*>(sw.cand_phat)[i] = valid ? phat_word(fph[f] * w.rprob[src]) : ~0ull;
+        reinterpret_cast<unsigned int*>(sw.cand_tok)[i] = valid ? (0x80000000u | (unsigned int)tok) : ~0u;
+    }
+    __syncthreads();
+    const bool small = N <= 1024;
+    if (tt < 32 && small) { stage_layer_candidates(ls, sw, fsize, p.k); cp_async_wait_all(); }
+    if (tt == 0) {
+        LayerJob& j = ls.job;
+        j.kind = 1; j.d = d; j.fsize = fsize; j.n = p.n; j.k = p.k; j.kk = p.kk;
+        j.cand_phat = sw.cand_phat; j.cand_tok = sw.cand_tok;
+        j.T_tok = sw.T_tok; j.T_par = sw.T_par; j.T_phat = sw.T_phat;
+        j.fmap = nullptr; j.nR_old = 0; j.off = 0; j.Rnew = nullptr;
+    }
+    __syncthreads();
+    const LayerJob j = ls.job;
+    const int nl = small ? select_layer_team<false>(ls, j, tt, w.status) : select_layer_team_big<false>(ls, j, tt, w.status);
+    if (tt >= 32) return;                                    // the rest is one warp's work
+    const bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta, w.status);
+    if (more) {
+        const int gid0 = (d - 1) * p.n;
+        for (int i = lane; i < nl; i += 32) {
+            next_tokens[(size_t)b * p.n + i] = ls.ltok[i];
+            next_parent[(size_t)b * p.n + i] = __ldcg(&sw.T_par[gid0 + i]);
+            w.front_phat[(size_t)b * p.n + i] = __longlong_as_double((long long)(ls.lkeys[i] - 1ull));
+        }
+        if (lane == 0) { sw.st[kStDepth] = d + 1; sw.st[kStFsize] = nl; next_count[b] = nl; }
+    } else if (lane == 0) {
+        sw.st[kStDepth] = 0; next_count[b] = 0;
+    }
 }
 
 // Tree attention mask + position ids: one CTA per sequence, one thread per node.
@@ -925,6 +1003,36 @@ int opt_tree_post_verify(opt_tree_ctx* ctx, const opt_tree_out* tree, const uint
                  tree->n_sel, mask, accept_len, accept_nodes, ctx->cfg.n, ctx->cfg.max_depth, dense_mask, kv_gather, kv_keep,
                  ctx->ws.status);
     ctx->launches++;
+    return check_launch();
+}
+
+int opt_tree_layers_begin(opt_tree_ctx* ctx, int32_t B, void* stream) {
+    if (!ctx || B < 1 || B > ctx->cfg.max_batch) return OPT_TREE_ERR_INVALID_ARG;
+    ot::Params p = make_params(ctx, nullptr, 0.0f);
+    p.B = B;
+    launch_after(ot::layers_begin_kernel, dim3((unsigned)((B + 127) / 128)), dim3(128), 0, static_cast<cudaStream_t>(stream), ctx->ws, p);
+    ctx->launches++;
+    return check_launch();
+}
+
+int opt_tree_layers_step(opt_tree_ctx* ctx, const void* frontier_logits, int32_t frontier_stride, int32_t B, float delta,
+                         const opt_tree_out* out, int32_t* next_tokens, int32_t* next_parent, int32_t* next_count, void* stream) {
+    if (!ctx || !frontier_logits || bad_tree(out) || !next_tokens || !next_parent || !next_count || B < 1 ||
+        B > ctx->cfg.max_batch || frontier_stride < 1 || frontier_stride > ctx->cfg.n || delta != delta)
+        return OPT_TREE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ot::Params p = make_params(ctx, frontier_logits, delta);
+    p.B = B;
+    const int nrows = B * frontier_stride;
+    ot::Params pr = p;
+    pr.H = nrows;                                            // the dense buffer is the "table" of the row step
+    const int grid = nrows < ctx->grid ? nrows : ctx->grid;
+    launch_after(ot::row_topk_kernel, dim3(grid), dim3(ot::kThreads), sizeof(ot::CtaSmem), st,
+                 pr, static_cast<const uint16_t*>(frontier_logits), static_cast<const int32_t*>(nullptr), nrows, ctx->ws.rtok,
+                 ctx->ws.rprob, ctx->ws.status);
+    launch_after(ot::layer_step_kernel, dim3(B), dim3(ot::kTeam), 0, st, ctx->ws, p, frontier_stride, *out, next_tokens,
+                 next_parent, next_count);
+    ctx->launches += 2;
     return check_launch();
 }
 

@@ -120,7 +120,7 @@ struct SeqWork {
     int32_t* st;           // [8]      1: rows finished since the build began, 2: |R|, 3: rows sent out in all
     int32_t* fmap;         // [n]      pruned draft: layer slot of the node behind each frontier row
 };
-enum { kStDone = 1, kStNR = 2, kStRows = 3 };
+enum { kStDone = 1, kStNR = 2, kStRows = 3, kStDepth = 4, kStFsize = 5 };   // 4, 5: layer-by-layer build: layer awaited (0: finished), its rows
 
 struct TreeOut {           // mirrors opt_tree_out, pointers offset to the sequence
     int32_t *token, *parent, *depth;
