@@ -206,7 +206,7 @@ __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restri
     if (i < p.B) {
         int32_t* st = w.st + (size_t)i * 8;
         st[kStDone] = 0; st[kStNR] = 0; st[kStRows] = 0;
-        w.fmap[(size_t)i * p.n] = 0;                                      // the root row stands for "slot 0"
+        for (int f = 0; f < p.n; ++f) w.fmap[(size_t)i * p.n + f] = f;    // frontier row f stands for layer slot f unless a pruned layer says otherwise
         w.E_prev[i] = 0.0;
     }
     if (i == 0) { w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; w.q_ctl[kQCursor] = p.B; }   // the roots are rows 0 .. B-1
@@ -385,7 +385,7 @@ struct BuildSink {
             team_sync();
             const LayerJob j = ls.job;
             if (j.kind == 0) return;
-            if (kPrune && j.kind == 2) select_running_team(ls, j, tt, w.status);
+            if (j.kind == 2) select_running_team(ls, j, tt, w.status);
             else if (j.fsize * j.k <= 1024) select_layer_team<kPrune>(ls, j, tt, w.status);
             else select_layer_team_big<kPrune>(ls, j, tt, w.status);
         }
@@ -419,13 +419,16 @@ struct BuildSink {
                     const int nvalid = fsize * p.kk, nl = nvalid < p.n ? nvalid : p.n;
                     // Without a threshold the loop test only looks at the depth: the next layer's rows
                     // can go out before the running top-n is brought up to date.
-                    if (kPrune) {
+                    // The pruned draft always takes the one-selection layer job; the ordinary build takes it for
+                    // the layer at the depth limit, after which nothing is drafted: the nodes of that layer that
+                    // do not reach the running top-n need not be stored, and one selection does instead of two.
+                    if (kPrune || d == p.Dcap) {
                         const int nR_old = d == 1 ? 0 : __ldcg(&sw.st[kStNR]);
                         const int off = (nR_old + 1) & ~1;
                         if (off + fsize * p.k <= 1024) {
                             const int sent = merged_layer_job(ls, sw, b, d, fsize, nR_old, off);
                             if (sent > 0) { cur_d[q] = d + 1; cur_f[q] = sent; cur_tot[q] += sent; }
-                            if (lane == 0) sw.st[kStRows] = cur_tot[q];
+                            if (kPrune && lane == 0) sw.st[kStRows] = cur_tot[q];
                             if (sent <= 0) {
                                 cur_d[q] = 0; --live;
                                 __threadfence();
@@ -458,7 +461,7 @@ struct BuildSink {
                     if (early) publish_layer(ls, b, d, nl, g0);
                     bool more = update_running_warp(ls, sw, tree_out(out, p, b), d, nl, p.n, p.Dcap, p.max_depth, p.delta,
                                                     w.status);
-                    if (kPrune && lane == 0) { ls.cache_b = b; ls.cache_d = d; }     // rsel / vals now hold this top-n
+                    if (lane == 0) { ls.cache_b = b; ls.cache_d = d; }                // rsel / vals now hold this top-n
                     int sent = nl;                             // rows of the next layer
                     if (kPrune && more) {
                         // The new layer's nodes among the n largest are the tail of the ascending list rsel
