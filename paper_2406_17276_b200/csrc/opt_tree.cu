@@ -203,10 +203,11 @@ __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restri
         reinterpret_cast<unsigned long long*>(w.cand_phat)[j] = 0ull;
         w.cand_tok[j] = 0;
     }
+    // frontier row f stands for layer slot f unless a pruned layer says otherwise
+    for (long long j = i; j < (long long)p.B * p.n; j += (long long)gridDim.x * blockDim.x) w.fmap[j] = (int32_t)(j % p.n);
     if (i < p.B) {
         int32_t* st = w.st + (size_t)i * 8;
         st[kStDone] = 0; st[kStNR] = 0; st[kStRows] = 0;
-        for (int f = 0; f < p.n; ++f) w.fmap[(size_t)i * p.n + f] = f;    // frontier row f stands for layer slot f unless a pruned layer says otherwise
         w.E_prev[i] = 0.0;
     }
     if (i == 0) { w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; w.q_ctl[kQCursor] = p.B; }   // the roots are rows 0 .. B-1
