@@ -192,6 +192,46 @@ def mask_of(parent, depth, n_sel: int, n: int, base_pos: int = 0):
     return mask, pos
 
 
+def philox4x32_10(ctr, key):
+    """The generator's block function: 4 x uint32 counter, 2 x uint32 key -> 4 x uint32."""
+    c = np.ascontiguousarray(ctr, np.uint32); k = np.ascontiguousarray(key, np.uint32); o = np.zeros(4, np.uint32)
+    lib().ot_philox4x32_10(_p(c, C.c_uint32), _p(k, C.c_uint32), _p(o, C.c_uint32))
+    return o
+
+
+def uniform(seed: int, step: int, sequence: int, position: int) -> float:
+    lib().ot_uniform.restype = C.c_double
+    return float(lib().ot_uniform(C.c_uint64(seed), C.c_uint64(step), C.c_int32(sequence), C.c_int32(position)))
+
+
+def sample_token(x: np.ndarray, tau: float, u: float):
+    """(token, margin) of one inverse-CDF sample of softmax(x / tau)."""
+    x = np.ascontiguousarray(x, np.float64)
+    mg = C.c_double()
+    lib().ot_sample_token.restype = C.c_int32
+    y = lib().ot_sample_token(_p(x, C.c_double), C.c_int32(x.shape[0]), C.c_double(tau), C.c_double(u), C.byref(mg))
+    return int(y), mg.value
+
+
+def table_verify_sampled(target: np.ndarray, root_token, token, parent, depth, n_sel, max_depth: int, tau: float, seed: int, step: int):
+    """Sampled verification of a batch of packed trees on the table model."""
+    H, V = target.shape
+    root_token = np.ascontiguousarray(root_token, np.int32)
+    token = np.ascontiguousarray(token, np.int32); parent = np.ascontiguousarray(parent, np.int32)
+    depth = np.ascontiguousarray(depth, np.int32); n_sel = np.ascontiguousarray(n_sel, np.int32)
+    B, n = token.shape
+    out = dict(accept_len=np.zeros(B, np.int32), accept_tokens=np.full((B, max_depth + 1), -1, np.int32),
+               accept_nodes=np.full((B, max_depth), -1, np.int32), next_root=np.full(B, -1, np.int32),
+               min_margin=np.zeros(B, np.float64))
+    lib().ot_table_verify_sampled(
+        _p(target, C.c_uint16), C.c_int32(H), C.c_int32(V), _p(root_token, C.c_int32), C.c_int32(B), C.c_int32(n),
+        C.c_int32(max_depth), _p(token, C.c_int32), _p(parent, C.c_int32), _p(depth, C.c_int32), _p(n_sel, C.c_int32),
+        C.c_double(tau), C.c_uint64(seed), C.c_uint64(step),
+        _p(out["accept_len"], C.c_int32), _p(out["accept_tokens"], C.c_int32), _p(out["accept_nodes"], C.c_int32),
+        _p(out["next_root"], C.c_int32), _p(out["min_margin"], C.c_double))
+    return out
+
+
 def dense_mask_of(parent, n_sel: int, n: int) -> np.ndarray:
     """[n+1][n+1] uint8: who attends to whom inside one step (position 0 = root, i+1 = node i)."""
     parent = np.ascontiguousarray(parent, np.int32)

@@ -540,6 +540,129 @@ int32_t ot_verify(const ot_model *target, int32_t root_token, int32_t V, int32_t
 }
 
 /* ------------------------------------------------------------------------- */
+/* Verification with sampling (temperature > 0).  The paper evaluates it      */
+/* (the table with temperature 1) but says only that the acceptable tokens   */
+/* change; the rule here is this build's reading: at every visited position  */
+/* the next token is SAMPLED from the target's distribution at temperature   */
+/* tau, softmax(x / tau), and accepted as the walk's next token; the walk    */
+/* goes on while the current node has a child that carries the sampled       */
+/* token.  The emitted tokens are then exactly a sample of the target model, */
+/* and A = matched nodes + 1 as in the greedy walk.                          */
+/* Randomness: one uniform per (sequence, step position), from the counter-  */
+/* based generator Philox4x32-10 (Salmon et al., "Parallel random numbers:   */
+/* as easy as 1, 2, 3", 2011): key = the 64-bit seed, counter = (position,   */
+/* sequence, decoding step low, decoding step high); position 0 is the root, */
+/* position i+1 packed node i.  u = (53 top bits of the first two outputs) * */
+/* 2^-53.  Sampling is by inverse CDF in token order: with e_v = exp((x_v -  */
+/* max x) / tau) and S their sum in token order, the token is the first v    */
+/* whose running sum exceeds u * S (the last token with e_v > 0 if rounding  */
+/* leaves none).                                                             */
+/* ------------------------------------------------------------------------- */
+static void philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr_in[0], c1 = ctr_in[1], c2 = ctr_in[2], c3 = ctr_in[3];
+    uint32_t k0 = key_in[0], k1 = key_in[1];
+    for (int round = 0; round < 10; ++round) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+void ot_philox4x32_10(const uint32_t *ctr, const uint32_t *key, uint32_t *out) { philox4x32_10(ctr, key, out); }
+
+double ot_uniform(uint64_t seed, uint64_t step, int32_t sequence, int32_t position)
+{
+    uint32_t ctr[4] = { (uint32_t)position, (uint32_t)sequence, (uint32_t)step, (uint32_t)(step >> 32) };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) }, o[4];
+    philox4x32_10(ctr, key, o);
+    uint64_t bits = (((uint64_t)o[1] << 32) | o[0]) >> 11;
+    return (double)bits * (1.0 / 9007199254740992.0);
+}
+
+/* One sample; margin (if given) = distance of u*S from the nearer of the two running sums that
+ * bracket the chosen token, relative to S: a summation in another order may choose a neighbour
+ * only if this is at rounding level. */
+int32_t ot_sample_token(const double *x, int32_t V, double tau, double u, double *margin)
+{
+    double m = -INFINITY, S = 0.0;
+    for (int32_t v = 0; v < V; ++v) if (x[v] > m) m = x[v];
+    for (int32_t v = 0; v < V; ++v) S += exp((x[v] - m) / tau);
+    const double t = u * S;
+    double run = 0.0, before = 0.0;
+    int32_t last = 0, y = -1;
+    for (int32_t v = 0; v < V; ++v) {
+        double e = exp((x[v] - m) / tau);
+        if (e > 0.0) last = v;
+        before = run;
+        run += e;
+        if (run > t) { y = v; break; }
+    }
+    if (y < 0) { y = last; before = run; }
+    if (margin) {
+        double a = fabs(t - before), b = fabs(run - t);
+        *margin = (a < b ? a : b) / S;
+    }
+    return y;
+}
+
+int32_t ot_verify_sampled(const ot_model *target, int32_t root_token, int32_t V, int32_t n_sel, int32_t max_depth,
+                          const int32_t *token, const int32_t *parent, const int32_t *depth,
+                          double tau, uint64_t seed, uint64_t step, int32_t sequence,
+                          int32_t *accept_tokens, int32_t *accept_nodes, int32_t *next_root, double *min_margin)
+{
+    double *scratch = (double *)malloc((size_t)V * sizeof(double));
+    int32_t *path = (int32_t *)malloc((size_t)(max_depth + 1) * sizeof(int32_t));
+    for (int32_t i = 0; i <= max_depth; ++i) accept_tokens[i] = -1;
+    for (int32_t i = 0; i < max_depth; ++i) accept_nodes[i] = -1;
+    int32_t cur = -1, A = 0, curdepth = 0;
+    double mm = INFINITY;
+    for (;;) {
+        if (cur >= 0)
+            for (int32_t a = cur, i = curdepth - 1; a >= 0; a = parent[a], --i) path[i] = token[a];
+        target->logits(target->user, root_token, path, curdepth, scratch);
+        double mg;
+        int32_t y = ot_sample_token(scratch, V, tau, ot_uniform(seed, step, sequence, cur + 1), &mg);
+        if (mg < mm) mm = mg;
+        accept_tokens[A++] = y;
+        int32_t hit = -1;
+        for (int32_t i = 0; i < n_sel; ++i)
+            if (parent[i] == cur && token[i] == y) { hit = i; break; }
+        if (hit < 0) break;
+        accept_nodes[A - 1] = hit;
+        cur = hit;
+        curdepth = depth[hit];
+    }
+    *next_root = accept_tokens[A - 1];
+    if (min_margin) *min_margin = mm;
+    free(scratch); free(path);
+    return A;
+}
+
+/* Sampled verification of a batch on the table model. */
+int ot_table_verify_sampled(const uint16_t *target, int32_t H, int32_t V, const int32_t *root_token, int32_t batch,
+                            int32_t n, int32_t max_depth, const int32_t *token, const int32_t *parent, const int32_t *depth,
+                            const int32_t *n_sel, double tau, uint64_t seed, uint64_t step,
+                            int32_t *accept_len, int32_t *accept_tokens, int32_t *accept_nodes, int32_t *next_root,
+                            double *min_margin)
+{
+    ot_table_model tm = { target, H, V };
+    ot_model tmodel = { ot_table_logits, ot_table_key, &tm };
+    for (int32_t b = 0; b < batch; ++b)
+        accept_len[b] = ot_verify_sampled(&tmodel, root_token[b], V, n_sel[b], max_depth,
+                                          token + (size_t)b * n, parent + (size_t)b * n, depth + (size_t)b * n,
+                                          tau, seed, step, b,
+                                          accept_tokens + (size_t)b * (max_depth + 1), accept_nodes + (size_t)b * max_depth,
+                                          next_root + b, min_margin ? min_margin + b : NULL);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Batch driver over the table model (what the harness times and compares).  */
 /* One decoding step for `batch` independent sequences, single thread.       */
 /* All per-sequence outputs are [batch][...] contiguous.                     */
