@@ -187,6 +187,23 @@ int opt_tree_layers_step(opt_tree_ctx *ctx, const void *frontier_logits_bf16, in
                          float delta, const opt_tree_out *out, int32_t *next_tokens, int32_t *next_parent,
                          int32_t *next_count, void *stream);
 
+/* Verification with sampling at temperature tau > 0.  The paper evaluates a temperature of 1 and says
+ * only that the acceptable tokens change; this library's rule: at every position of the walk the next
+ * token is drawn from the target's distribution softmax(x / tau) and accepted, and the walk goes on
+ * while the current node has a child that carries the drawn token.  The emitted tokens are thus a
+ * sample of the target model; outputs are those of opt_tree_verify.
+ * Randomness is reproducible: one uniform per (sequence b, position j; 0 = root, i+1 = node i) from the
+ * counter-based generator Philox4x32-10 (Salmon et al., 2011) with key = seed and counter =
+ * (j, b, step low word, step high word), u = top 53 bits of the first two output words * 2^-53; the
+ * draw is by inverse CDF in token order on e_v = exp((x_v - max x) / tau) in double precision (the
+ * first token whose running sum exceeds u * sum; the last token with e_v > 0 if rounding leaves none).
+ * `step` is the caller's decoding step number, so that successive steps use fresh uniforms.
+ * Errors as opt_tree_verify; tau <= 0 or NaN is OPT_TREE_ERR_INVALID_ARG. */
+int opt_tree_verify_sampled(opt_tree_ctx *ctx, const opt_tree_out *tree, const void *target_logits_bf16,
+                            const int32_t *root_token, int32_t B, double tau, uint64_t seed, uint64_t step,
+                            int32_t *accept_len, int32_t *accept_tokens, int32_t *accept_nodes,
+                            int32_t *next_root, void *stream);
+
 /* Bookkeeping after verification (Algorithm 2: the mask that M(T_opt, mask) consumes, in dense
  * form; Section 3, last paragraph: both models keep key and value caches, so after Verify only
  * the accepted tokens' entries stay).  The paper fixes neither format; this library's are:

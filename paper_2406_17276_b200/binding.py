@@ -20,7 +20,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -
 EXPORTS = ["opt_tree_workspace_bytes", "opt_tree_create", "opt_tree_destroy", "opt_tree_build", "opt_tree_mask",
            "opt_tree_verify", "opt_tree_row_softmax_topk", "opt_tree_step_host", "opt_tree_last_device_status",
            "opt_tree_launch_count", "opt_tree_strerror", "opt_tree_verify_static", "opt_tree_post_verify", "opt_tree_build_pruned", "opt_tree_layers_begin",
-           "opt_tree_layers_step"]
+           "opt_tree_layers_step", "opt_tree_verify_sampled"]
 
 
 class Config(C.Structure):
@@ -68,6 +68,8 @@ def lib():
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.opt_tree_build_pruned.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_float, C.POINTER(Out), C.c_void_p,
                                             C.c_void_p]
+        L.opt_tree_verify_sampled.argtypes = [C.c_void_p, C.POINTER(Out), C.c_void_p, C.c_void_p, C.c_int32, C.c_double,
+                                              C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.opt_tree_layers_begin.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
         L.opt_tree_layers_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.POINTER(Out), C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_void_p]
@@ -218,6 +220,19 @@ class OptTree:
         cs = tree.c_struct()
         _check(lib().opt_tree_post_verify(self._ctx, C.byref(cs), _ptr(mask), _ptr(accept_len), _ptr(accept_nodes), B,
                                           _ptr(out[0]), _ptr(out[1]), _ptr(out[2]), _stream()), "opt_tree_post_verify")
+        return out
+
+    def verify_sampled(self, tree: Tree, target: torch.Tensor, root_token: torch.Tensor, tau: float, seed: int, step: int,
+                       out=None):
+        B = tree.token.shape[0]
+        D = self.cfg.max_depth
+        if out is None:
+            i32 = dict(dtype=torch.int32, device=self.device)
+            out = (torch.empty(B, **i32), torch.empty((B, D + 1), **i32), torch.empty((B, D), **i32), torch.empty(B, **i32))
+        cs = tree.c_struct()
+        _check(lib().opt_tree_verify_sampled(self._ctx, C.byref(cs), _ptr(target), _ptr(root_token), B, C.c_double(tau),
+                                             C.c_uint64(seed), C.c_uint64(step), _ptr(out[0]), _ptr(out[1]), _ptr(out[2]),
+                                             _ptr(out[3]), _stream()), "opt_tree_verify_sampled")
         return out
 
     def row_softmax_topk(self, logits: torch.Tensor, rows: torch.Tensor):

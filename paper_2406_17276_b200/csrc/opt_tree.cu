@@ -710,6 +710,51 @@ struct VerifySmem {
     int hit;
 };
 
+// The end of a verification CTA: position j's token y is recorded; the CTA that records a sequence's
+// last token walks the tree: accept the child that carries the recorded token, until none does.
+__device__ void verify_tail(VerifySmem& s, const Workspace& w, const Params& p, int b, int j, int ns, int y,
+                            const int32_t* tok, const int32_t* par, int32_t* accept_len, int32_t* accept_tokens,
+                            int32_t* accept_nodes, int32_t* next_root) {
+    const int tid = threadIdx.x;
+    int32_t* g = w.g + (size_t)b * (p.n + 1);
+    if (tid == 0) {
+        g[j] = y;
+        __threadfence();
+        s.flag = (atomicAdd(&w.vdone[b], 1) == ns);
+    }
+    __syncthreads();
+    if (!s.flag) return;
+    __threadfence();
+
+    // acceptance walk (block-wide child search; children of one node carry distinct tokens)
+    int32_t* at = accept_tokens + (size_t)b * (p.max_depth + 1);
+    int32_t* an = accept_nodes + (size_t)b * p.max_depth;
+    for (int i = tid; i <= p.max_depth; i += kVerifyThreads) at[i] = -1;
+    for (int i = tid; i < p.max_depth; i += kVerifyThreads) an[i] = -1;
+    __syncthreads();
+    int cur = -1, A = 0;
+    for (int step = 0; step <= p.max_depth; ++step) {
+        const int yy = __ldcg(&g[cur + 1]);
+        if (tid == 0) { at[A] = yy; s.hit = -1; }
+        ++A;
+        __syncthreads();
+        if (A > p.max_depth) break;
+        for (int i = tid; i < ns; i += kVerifyThreads)
+            if (par[i] == cur && tok[i] == yy) s.hit = i;
+        __syncthreads();
+        const int hit = s.hit;
+        __syncthreads();
+        if (hit < 0) break;
+        if (tid == 0) an[A - 1] = hit;
+        cur = hit;
+    }
+    if (tid == 0) {
+        accept_len[b] = A;
+        next_root[b] = __ldcg(&g[cur + 1]);
+        w.vdone[b] = 0;
+    }
+}
+
 // Greedy verification.  CTA (j, b): j = 0 takes the target row after the root, j >= 1 the row after
 // kept node j-1; each finds the row's argmax (lowest token on ties).  The last CTA of a sequence
 // then walks the tree: accept the child that carries the target's token, until none does.
@@ -766,44 +811,114 @@ verify_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const 
     best_key = warp_max_u64(best_key);
     if ((tid & 31) == 0) s.red_u64[tid >> 5] = best_key;
     __syncthreads();
-    int32_t* g = w.g + (size_t)b * (p.n + 1);
-    if (tid == 0) {
+    if (tid == 0)
         for (int q = 1; q < kVerifyThreads / 32; ++q) best_key = s.red_u64[q] > best_key ? s.red_u64[q] : best_key;
-        g[j] = (int32_t)cand_token(best_key);
-        __threadfence();
-        s.flag = (atomicAdd(&w.vdone[b], 1) == ns);
-    }
-    __syncthreads();
-    if (!s.flag) return;
-    __threadfence();
+    verify_tail(s, w, p, b, j, ns, (int32_t)cand_token(best_key), tok, par, accept_len, accept_tokens, accept_nodes, next_root);
+}
 
-    // acceptance walk (block-wide child search; children of one node carry distinct tokens)
-    int32_t* at = accept_tokens + (size_t)b * (p.max_depth + 1);
-    int32_t* an = accept_nodes + (size_t)b * p.max_depth;
-    for (int i = tid; i <= p.max_depth; i += kVerifyThreads) at[i] = -1;
-    for (int i = tid; i < p.max_depth; i += kVerifyThreads) an[i] = -1;
+// ------------------------------------------------------------------------------------------------
+// Verification with sampling (temperature tau > 0): at every position the next token is drawn from
+// softmax(x / tau) of the target row by inverse CDF in token order, with one uniform per (sequence,
+// position) from the counter-based generator Philox4x32-10 (Salmon et al. 2011; key = seed, counter =
+// (position, sequence, step low, step high)); the walk is the greedy one on the drawn tokens.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1,
+                                              uint32_t& o0, uint32_t& o1) {
+#pragma unroll 1
+    for (int round = 0; round < 10; ++round) {
+        const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+        const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+        const uint32_t n0 = h1 ^ c1 ^ k0, n2 = h0 ^ c3 ^ k1;
+        c0 = n0; c1 = l1; c2 = n2; c3 = l0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    o0 = c0; o1 = c1;
+}
+__device__ __forceinline__ double uniform53(unsigned long long seed, unsigned long long step, int sequence, int position) {
+    uint32_t o0, o1;
+    philox4x32_10((uint32_t)position, (uint32_t)sequence, (uint32_t)step, (uint32_t)(step >> 32), (uint32_t)seed,
+                  (uint32_t)(seed >> 32), o0, o1);
+    const unsigned long long bits = (((unsigned long long)o1 << 32) | o0) >> 11;
+    return (double)bits * (1.0 / 9007199254740992.0);
+}
+
+struct SampleSmem {
+    double wsum[kVerifyThreads / 32];
+    float wmax[kVerifyThreads / 32];
+    int chosen, last_live;
+};
+
+// CTA (j, b) as in verify_kernel.  Thread t owns the tokens [t*L, (t+1)*L): its own sum, a scan over the
+// threads in token order, and the thread in whose stretch u*S falls walks it once more.
+__global__ void __launch_bounds__(kVerifyThreads)
+verify_sampled_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const int32_t* __restrict__ root_token,
+                      opt_tree_out tree, double tau, unsigned long long seed, unsigned long long step, int32_t* accept_len,
+                      int32_t* accept_tokens, int32_t* accept_nodes, int32_t* next_root) {
+    __shared__ VerifySmem s;
+    __shared__ SampleSmem q;
+    grid_dependency_wait();
+    const int b = blockIdx.y, j = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
+    const int ns = tree.n_sel[b];
+    if (j > ns) return;
+    const int32_t* tok = tree.token + (size_t)b * p.n;
+    const int32_t* par = tree.parent + (size_t)b * p.n;
+    int token = j == 0 ? root_token[b] : tok[j - 1];
+    const int depth = j == 0 ? 0 : tree.depth[(size_t)b * p.n + j - 1];
+    if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
+    const uint16_t* row = target + (size_t)row_of(token, depth, p.H) * p.V;
+    const int L = (((p.V + kVerifyThreads - 1) / kVerifyThreads) + 7) & ~7;       // tokens per thread, a multiple of 8
+    const int lo = min(tid * L, p.V), hi = min(lo + L, p.V);
+    auto logit = [&](int v) -> float { return bf16_bits_to_float(__ldg(row + v)); };
+
+    // the row's maximum
+    float mx = -INFINITY;
+    for (int v = lo; v < hi; ++v) mx = fmaxf(mx, logit(v));
+    mx = warp_max_f32(mx);
+    if (lane == 0) q.wmax[wp] = mx;
+    if (tid == 0) { q.chosen = -1; q.last_live = -1; }
     __syncthreads();
-    int cur = -1, A = 0;
-    for (int step = 0; step <= p.max_depth; ++step) {
-        const int y = __ldcg(&g[cur + 1]);
-        if (tid == 0) { at[A] = y; s.hit = -1; }
-        ++A;
-        __syncthreads();
-        if (A > p.max_depth) break;
-        for (int i = tid; i < ns; i += kVerifyThreads)
-            if (par[i] == cur && tok[i] == y) s.hit = i;
-        __syncthreads();
-        const int hit = s.hit;
-        __syncthreads();
-        if (hit < 0) break;
-        if (tid == 0) an[A - 1] = hit;
-        cur = hit;
+    mx = q.wmax[0];
+#pragma unroll
+    for (int i = 1; i < kVerifyThreads / 32; ++i) mx = fmaxf(mx, q.wmax[i]);
+    const double m = (double)mx, inv_tau = 1.0 / tau;
+
+    // this thread's sum in token order, then the sums before it
+    double mine = 0.0;
+    int live = -1;                                           // last token of the stretch with a positive term
+    for (int v = lo; v < hi; ++v) {
+        const double e = exp(((double)logit(v) - m) / tau);
+        mine += e;
+        if (e > 0.0) live = v;
     }
-    if (tid == 0) {
-        accept_len[b] = A;
-        next_root[b] = __ldcg(&g[cur + 1]);
-        w.vdone[b] = 0;
+    (void)inv_tau;
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += up;
     }
+    if (lane == 31) q.wsum[wp] = incl;
+    __syncthreads();
+    double before = 0.0, S = 0.0;
+#pragma unroll
+    for (int i = 0; i < kVerifyThreads / 32; ++i) { const double x = q.wsum[i]; S += x; before += i < wp ? x : 0.0; }
+    incl += before;
+    const double excl = incl - mine;
+    const double t = uniform53(seed, step, b, j) * S;
+    atomicMax(&q.last_live, live);
+    if (incl > t && !(excl > t) && hi > lo) {                // the stretch in which the running sum passes t
+        double run = excl;
+        int y = live;
+        for (int v = lo; v < hi; ++v) {
+            run += exp(((double)logit(v) - m) / tau);
+            if (run > t) { y = v; break; }
+        }
+        atomicMax(&q.chosen, y);                             // (at most one thread gets here)
+    }
+    __syncthreads();
+    int y = q.chosen;
+    if (y < 0) y = q.last_live < 0 ? 0 : q.last_live;        // rounding left no stretch: the last token with a positive term
+    verify_tail(s, w, p, b, j, ns, y, tok, par, accept_len, accept_tokens, accept_nodes, next_root);
 }
 
 }  // namespace ot
@@ -993,6 +1108,20 @@ int opt_tree_verify(opt_tree_ctx* ctx, const opt_tree_out* tree, const void* tar
     const ot::Params p = make_params(ctx, target, 0.0f);
     launch_after(ot::verify_kernel, dim3(ctx->cfg.n + 1, B), dim3(ot::kVerifyThreads), 0, static_cast<cudaStream_t>(stream),
                  ctx->ws, p, static_cast<const uint16_t*>(target), root_token, *tree, accept_len, accept_tokens, accept_nodes, next_root);
+    ctx->launches++;
+    return check_launch();
+}
+
+int opt_tree_verify_sampled(opt_tree_ctx* ctx, const opt_tree_out* tree, const void* target, const int32_t* root_token, int32_t B,
+                            double tau, uint64_t seed, uint64_t step, int32_t* accept_len, int32_t* accept_tokens,
+                            int32_t* accept_nodes, int32_t* next_root, void* stream) {
+    if (!ctx || bad_tree(tree) || !target || !root_token || !accept_len || !accept_tokens || !accept_nodes || !next_root ||
+        B < 1 || B > ctx->cfg.max_batch || !(tau > 0.0))
+        return OPT_TREE_ERR_INVALID_ARG;
+    const ot::Params p = make_params(ctx, target, 0.0f);
+    launch_after(ot::verify_sampled_kernel, dim3(ctx->cfg.n + 1, B), dim3(ot::kVerifyThreads), 0, static_cast<cudaStream_t>(stream),
+                 ctx->ws, p, static_cast<const uint16_t*>(target), root_token, *tree, tau, (unsigned long long)seed,
+                 (unsigned long long)step, accept_len, accept_tokens, accept_nodes, next_root);
     ctx->launches++;
     return check_launch();
 }
