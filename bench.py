@@ -46,7 +46,7 @@ def _peaks():
 # capture, see profiles/), keyed by workload, with the digest of the kernel sources the counters
 # were taken on: a changed kernel reports no traffic.
 NCU_TRAFFIC = {
-    "c4": {"bytes": 594.7e6, "csrc_sha256": "8fb9fc6332e6947a080880bdf4e32d3fcb928167246e0b2e159c6bc0eb41479d"},
+    "c4": {"bytes": 596.4e6, "csrc_sha256": "ab0613a6d771ea85cb46a2d70e1e949059ee37d9f8bcb7188dde00c39560c10a"},
 }
 
 
@@ -281,6 +281,20 @@ def run_cuda(args):
             raise SystemExit("bench.py: device status after layers_step")
         del layer_bufs[:]
 
+    # ---- verification with sampling (temperature 1): timed on its own ----
+    sv_out = ot.verify_sampled(tree, d_lt, roots0, 1.0, 2024, 0)
+    for _ in range(3):
+        ot.verify_sampled(tree, d_lt, roots0, 1.0, 2024, 0, sv_out)
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    s0.record()
+    for i in range(50):
+        ot.verify_sampled(tree, d_lt, roots0, 1.0, 2024, i, sv_out)
+    s1.record(); torch.cuda.synchronize()
+    verify_sampled_us = s0.elapsed_time(s1) * 20.0
+    if ot.device_status() != 0:
+        raise SystemExit("bench.py: device status after verify_sampled")
+
     peak, peak_kind = _peaks()
     achieved = algo_bytes / (build_ms * 1e-3) / 1e9
     line = {
@@ -301,6 +315,8 @@ def run_cuda(args):
                          "note": "opt_tree_build_pruned alone on the first step's roots: the same trees, only rows that can still matter; not the benchmark's metric"},
         "layers_build": {"ms_per_batch": layers_ms, "trees_per_s": (B / (layers_ms * 1e-3)) if layers_ms else None,
                          "note": "opt_tree_layers_begin + one opt_tree_layers_step per layer on pre-gathered logits (two launches per layer; skipped when those logits would not fit); not the benchmark's metric"},
+        "verify_sampled": {"us_per_call": verify_sampled_us,
+                           "note": "opt_tree_verify_sampled alone at temperature 1 (one double-precision exponential per target logit, twice); not part of the timed step"},
         "post_verify": {"us_per_call": post_verify_us, "bytes_written": int(sum(t.numel() * t.element_size() for t in pv_out)),
                         "note": "opt_tree_post_verify alone, 100 back-to-back calls; not part of the timed step"},
         "roofline": {"bound": "hbm", "kernel": "build_kernel (opt_tree_build: init_build_kernel + one persistent build_kernel)",
