@@ -869,10 +869,20 @@ verify_sampled_kernel(Workspace w, Params p, const uint16_t* __restrict__ target
     const int L = (((p.V + kVerifyThreads - 1) / kVerifyThreads) + 7) & ~7;       // tokens per thread, a multiple of 8
     const int lo = min(tid * L, p.V), hi = min(lo + L, p.V);
     auto logit = [&](int v) -> float { return bf16_bits_to_float(__ldg(row + v)); };
+    const bool vec = p.aligned != 0;                         // then a stretch starts on a 16-byte boundary and V is a multiple of 8
+    const uint4* rv = reinterpret_cast<const uint4*>(row);
 
     // the row's maximum
     float mx = -INFINITY;
-    for (int v = lo; v < hi; ++v) mx = fmaxf(mx, logit(v));
+    if (vec) {
+        for (int v8 = lo >> 3; v8 < hi >> 3; ++v8) {
+            const uint4 x = ld_nc_v4(rv + v8);
+            const uint32_t m2 = max_bf16x2(max_bf16x2(x.x, x.y), max_bf16x2(x.z, x.w));
+            mx = fmaxf(mx, fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u)));
+        }
+    } else {
+        for (int v = lo; v < hi; ++v) mx = fmaxf(mx, logit(v));
+    }
     mx = warp_max_f32(mx);
     if (lane == 0) q.wmax[wp] = mx;
     if (tid == 0) { q.chosen = -1; q.last_live = -1; }
@@ -885,10 +895,24 @@ verify_sampled_kernel(Workspace w, Params p, const uint16_t* __restrict__ target
     // this thread's sum in token order, then the sums before it
     double mine = 0.0;
     int live = -1;                                           // last token of the stretch with a positive term
-    for (int v = lo; v < hi; ++v) {
-        const double e = exp(((double)logit(v) - m) / tau);
-        mine += e;
-        if (e > 0.0) live = v;
+    if (vec) {
+        for (int v8 = lo >> 3; v8 < hi >> 3; ++v8) {
+            const uint4 x = ld_nc_v4(rv + v8);
+            const uint32_t ww[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int e8 = 0; e8 < 8; ++e8) {
+                const uint32_t bits = (e8 & 1) ? (ww[e8 >> 1] >> 16) : (ww[e8 >> 1] & 0xFFFFu);
+                const double e = exp(((double)bf16_bits_to_float(bits) - m) / tau);
+                mine += e;
+                if (e > 0.0) live = v8 * 8 + e8;
+            }
+        }
+    } else {
+        for (int v = lo; v < hi; ++v) {
+            const double e = exp(((double)logit(v) - m) / tau);
+            mine += e;
+            if (e > 0.0) live = v;
+        }
     }
     (void)inv_tau;
     double incl = mine;
