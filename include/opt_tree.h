@@ -21,7 +21,7 @@
  *   - Logits must be finite or -inf (no NaN, no +inf); a row must hold at least one finite
  *     value.  Behaviour on other inputs is unspecified but never faults.
  *   - The root is not a node of the output, is not counted in n and has no mask bit
- *     (Section 3: "the root node is not considered when calculating node trees").
+ *     (Section 3, definition of E_sub: the root is left out of the node count).
  */
 #ifndef OPT_TREE_H_
 #define OPT_TREE_H_
@@ -81,7 +81,7 @@ size_t opt_tree_workspace_bytes(const opt_tree_config *cfg);
 int opt_tree_create(opt_tree_ctx **ctx, const opt_tree_config *cfg);
 int opt_tree_destroy(opt_tree_ctx *ctx);
 
-/* Algorithm 1 ("Construct an OPT-Tree") for B independent sequences.
+/* Algorithm 1 (construction of an OPT-Tree) for B independent sequences.
  *   draft_logits_bf16 (dev) [H][V]   16-byte aligned base
  *   root_token        (dev) [B]      last token x_l of each input sequence, 0 <= token < V
  *   delta                            threshold of the loop test (E_sub(T,n) - E > delta); pass
@@ -167,7 +167,7 @@ int opt_tree_build_pruned(opt_tree_ctx *ctx, const void *draft_logits_bf16, cons
                           int32_t B, float delta, const opt_tree_out *out, int32_t *rows_read, void *stream);
 
 /* Layer-by-layer build, for a caller that runs a real draft model: Algorithm 1 with the draft step
- * ("compute the next token distributions of the nodes in the last layer") left to the caller.
+ * (the next-token distributions of the last layer's nodes) left to the caller.
  * opt_tree_layers_begin starts B trees; every opt_tree_layers_step takes the logits of the nodes
  * that are to be expanded (first the root's, then each returned layer's), grows every tree by one
  * layer exactly as opt_tree_build does (row softmax + top-k, Eq. 2, the n best candidates, E_sub,

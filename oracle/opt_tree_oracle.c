@@ -13,7 +13,10 @@
  * sort on the same bytes, closed forms on constant and one-hot rows, exhaustive
  * search over all parent-closed node subsets on tiny vocabularies, a hand-computed
  * example of Eq. 2 / Eq. 3, Theorem 1, Theorem 2, the closure proof, and a
- * path-enumeration definition of the greedy acceptance length.
+ * path-enumeration definition of the greedy acceptance length.  The two outputs that the
+ * parity tests use to tell a near-tie from an error, min_gap and stop_margin, are pinned by
+ * the same hand example (every boundary worked out by hand), by constructed ties and gaps,
+ * and by a NumPy replay of the selections on small random tables.
  * Not pinned ("parity unpinned"): the value E(A) = 2.07 of the paper's Figure 2 and the
  * mean acceptance lengths of Tables 1-3, which need the missing figure / real models.
  *
@@ -244,7 +247,8 @@ static int cmp_canon(const void *a, const void *b)
 
 static double rel_gap(double kept, double dropped)
 {
-    /* relative distance between the last kept and the first dropped value */
+    /* relative distance between the last kept and the first dropped value.  Path values are never
+     * negative and dropped <= kept, so kept == 0 means both are zero: an exact tie, gap 0. */
     double d = kept - dropped;
     if (kept <= 0.0) return 0.0;
     return d / kept;
@@ -442,10 +446,10 @@ int ot_table_build_rows(const uint16_t *draft, int32_t H, int32_t V, const int32
 }
 
 /* ------------------------------------------------------------------------- */
-/* Tree attention mask and position ids (Algorithm 2, "compute the           */
-/* corresponding tree attention mask"; Figure 1: nodes of a layer share the  */
-/* position index).  Row i has bit j set iff node j is i or an ancestor of i;*/
-/* W = ceil(n/64) words per row, bit j in word j/64 at position j%64.        */
+/* Tree attention mask and position ids (Algorithm 2, second line: the mask  */
+/* of T_opt; Figure 1: nodes of a layer share the position index).           */
+/* Row i has bit j set iff node j is i or an ancestor of i; W = ceil(n/64)   */
+/* words per row, bit j in word j/64 at position j%64.                       */
 /* ------------------------------------------------------------------------- */
 void ot_mask(const int32_t *parent, const int32_t *depth, int32_t n_sel, int32_t n, int32_t base_pos,
              uint64_t *mask, int32_t *position_ids)

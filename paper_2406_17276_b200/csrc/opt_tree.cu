@@ -1302,10 +1302,13 @@ int static_scratch(int32_t** out) {
 extern "C" int opt_tree_verify_static(const opt_tree_config* cfg, const opt_tree_out* tree, const void* target,
                                       const int32_t* root_token, int32_t B, int32_t* accept_len, int32_t* accept_tokens,
                                       int32_t* accept_nodes, int32_t* next_root, int32_t* device_status, void* stream) {
-    if (!valid_cfg(cfg) || bad_tree(tree) || !target || !root_token || !accept_len || !accept_tokens || !accept_nodes ||
+    if (!cfg) return OPT_TREE_ERR_INVALID_ARG;
+    opt_tree_config sized = *cfg;
+    sized.max_batch = 1;                                     // this entry point does not look at max_batch
+    if (!valid_cfg(&sized) || bad_tree(tree) || !target || !root_token || !accept_len || !accept_tokens || !accept_nodes ||
         !next_root || B < 1)
         return OPT_TREE_ERR_INVALID_ARG;
-    if (supported_cfg(cfg) != OPT_TREE_OK) return OPT_TREE_ERR_UNSUPPORTED;
+    if (supported_cfg(&sized) != OPT_TREE_OK) return OPT_TREE_ERR_UNSUPPORTED;
     if (B > OPT_TREE_STATIC_MAX_BATCH || cfg->n > OPT_TREE_STATIC_MAX_N) return OPT_TREE_ERR_UNSUPPORTED;
     int32_t* base = nullptr;
     const int rc = static_scratch(&base);

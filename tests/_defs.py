@@ -120,3 +120,42 @@ def target_chain(table, root_token, length):
         chain.append(y)
         tok, dep = y, dep + 1
     return chain
+
+
+def beam_boundaries(table, root_token, n, k, D, delta):
+    """The boundaries Algorithm 1 decides at, replayed with NumPy sorts on the nodes of full_tree.
+
+    Per drafted layer: the relative gap (kept - dropped) / kept between the last candidate that
+    enters the layer and the best one that does not, the same gap for the n largest nodes of T,
+    and |gain - delta| of every loop test that is evaluated.  Returns (smallest gap or inf,
+    smallest margin or inf, layers drafted).
+    """
+    D = min(D, n)
+    nodes = full_tree(table, root_token, k, D)            # (path, phat, parent index), breadth first
+    kids = {}
+    for i, (path, ph, par) in enumerate(nodes):
+        kids.setdefault(par, []).append(i)                # in sibling-rank order
+    gap, margin, E, T, layer = np.inf, np.inf, 0.0, [], [-1]
+    d = 0
+    while True:
+        d += 1
+        cand = [c for f in layer for c in kids.get(f, [])]          # candidate-index order
+        ph = np.array([nodes[c][1] for c in cand])
+        order = np.lexsort((np.arange(len(cand)), -ph))
+        nl = min(n, len(cand))
+        if len(cand) > nl:
+            gap = min(gap, (ph[order[nl - 1]] - ph[order[nl]]) / ph[order[nl - 1]])
+        layer = [cand[i] for i in sorted(order[:nl])]
+        T += layer
+        tp = np.sort(np.array([nodes[i][1] for i in T]))[::-1]
+        nR = min(n, len(T))
+        if len(T) > nR:
+            gap = min(gap, (tp[nR - 1] - tp[nR]) / tp[nR - 1])
+        esub = float(tp[:nR].sum())
+        if d >= D:
+            break
+        margin = min(margin, abs((esub - E) - delta))
+        if not (esub - E > delta):
+            break
+        E = esub
+    return gap, margin, d

@@ -8,22 +8,22 @@ import torch
 import oracle
 from paper_2406_17276_b200 import binding, synth
 from tests import _compare
-from tests._gpu import dev_table
+from tests._gpu import dev_table, poisoned_tree, record_parity
 
 pytestmark = pytest.mark.gpu
 NEG_INF = -math.inf
 FIELDS = ("token", "parent", "depth", "phat", "n_sel", "depth_reached", "expected_len", "esub_trace")
 
 
-def _run(w, delta, H=None, V=None, check_oracle=True):
+def _run(w, delta, H=None, V=None, check_oracle=True, test_id=None):
     ld, lt = synth.make_tables(w, H=H, V=V)
     Hh, Vv = ld.shape
     ot = binding.OptTree(Vv, Hh, w.n, w.k, w.max_depth, w.batch)
     d_ld = dev_table(ld)
     roots = synth.root_tokens(w.batch, Vv, w.seed + 4)
     r = torch.from_numpy(roots).cuda()
-    full = ot.build(d_ld, r, delta)
-    pruned, rows = ot.build_pruned(d_ld, r, delta)
+    full = ot.build(d_ld, r, delta, poisoned_tree(ot, w.batch))
+    pruned, rows = ot.build_pruned(d_ld, r, delta, poisoned_tree(ot, w.batch), torch.full((w.batch,), -1, dtype=torch.int32, device="cuda"))
     torch.cuda.synchronize()
     assert ot.device_status() == 0
     for f in FIELDS:                                   # the two device builds agree bit for bit
@@ -36,6 +36,9 @@ def _run(w, delta, H=None, V=None, check_oracle=True):
         g.update(mask=mask.cpu().numpy(), position_ids=pos.cpu().numpy())
         o, st = _compare.compare_step(w, ld, lt, roots, delta, g, check_verify=False)
         _, want_rows = oracle.table_build_rows(ld, roots, w.n, w.k, w.max_depth, delta, prune=True)
+        if test_id:
+            record_parity(f"{test_id}[{delta}]", st)
+        assert st["exact"] > 0 and st["near_tie"] + st["stop_near_tie"] <= 0.05 * (st["exact"] + 1)
         exact = st["near_tie"] == 0 and st["stop_near_tie"] == 0
         if exact:                                      # a tie broken the other way may change which rows are read
             assert np.array_equal(rows, want_rows), (rows, want_rows)
@@ -44,21 +47,21 @@ def _run(w, delta, H=None, V=None, check_oracle=True):
 
 @pytest.mark.parametrize("name,V,H", [("c1", 20000, 512), ("c2", 20000, 512), ("c4", 20000, 512), ("c3", 40008, 128), ("c5", 40008, 128)])
 @pytest.mark.parametrize("delta", [NEG_INF, 0.0, 0.2])
-def test_reduced_tables(name, V, H, delta):
-    _run(synth.WORKLOADS[name], delta, H=H, V=V)
+def test_reduced_tables(request, name, V, H, delta):
+    _run(synth.WORKLOADS[name], delta, H=H, V=V, test_id=request.node.nodeid)
 
 
 @pytest.mark.parametrize("n,k,D,B,V", [(1, 4, 5, 3, 512), (6, 1, 6, 3, 512), (256, 32, 20, 2, 4096), (5, 8, 3, 4, 8),
                                        (7, 3, 4, 2, 12), (10, 10, 6, 5, 100), (8, 4, 4, 300, 512)])
-def test_edge_sizes(n, k, D, B, V):
+def test_edge_sizes(request, n, k, D, B, V):
     w = synth.Workload("edge", B, V, n, k, D, 3.0, 1.1, 0.3, H=64, seed=n * 1000 + k)
     for delta in (NEG_INF, 0.1):
-        _run(w, delta)
+        _run(w, delta, test_id=request.node.nodeid)
 
 
-def test_full_size_c4_reads_fewer_rows():
+def test_full_size_c4_reads_fewer_rows(request):
     w = synth.WORKLOADS["c4"]
-    rows = _run(w, NEG_INF)
+    rows = _run(w, NEG_INF, test_id=request.node.nodeid)
     full_rows = w.batch * (1 + min(w.n, w.k) + (w.max_depth - 2) * w.n)
     assert rows.sum() < 0.5 * full_rows
 

@@ -7,13 +7,13 @@ import torch
 
 import oracle
 from paper_2406_17276_b200 import binding, synth
-from tests._gpu import dev_table
+from tests._gpu import dev_table, poisoned_verify_out, record_parity
 
 pytestmark = pytest.mark.gpu
 MARGIN = 1e-11        # a draw may fall the other way only where u*S sits this close (relative to S) to a running sum
 
 
-def _run(w, taus, H=None, V=None, steps=2):
+def _run(w, taus, H=None, V=None, steps=2, test_id=None):
     ld, lt = synth.make_tables(w, H=H, V=V)
     Hh, Vv = ld.shape
     ot = binding.OptTree(Vv, Hh, w.n, w.k, w.max_depth, w.batch)
@@ -24,7 +24,7 @@ def _run(w, taus, H=None, V=None, steps=2):
         r = torch.from_numpy(roots).cuda()
         tree = ot.build(d_ld, r, -math.inf)
         for step in range(steps):
-            al, at, an, nr = ot.verify_sampled(tree, d_lt, r, tau, 1234, step)
+            al, at, an, nr = ot.verify_sampled(tree, d_lt, r, tau, 1234, step, poisoned_verify_out(ot, w.batch))
             torch.cuda.synchronize()
             assert ot.device_status() == 0
             o = oracle.table_verify_sampled(lt, roots, tree.token.cpu().numpy(), tree.parent.cpu().numpy(), tree.depth.cpu().numpy(),
@@ -37,22 +37,24 @@ def _run(w, taus, H=None, V=None, steps=2):
                 else:
                     assert o["min_margin"][b] < MARGIN, (b, tau, step, o["min_margin"][b], g["accept_tokens"][b], o["accept_tokens"][b])
                     near += 1
+    if test_id:
+        record_parity(test_id, dict(exact=exact, near_tie=near, stop_near_tie=0, max_phat_rel=0.0, max_elen_rel=0.0))
     assert exact > 0 and near <= 0.02 * (exact + 1)
     return exact, near
 
 
 @pytest.mark.parametrize("name,V,H", [("c1", 20000, 256), ("c4", 8200, 128), ("c2", 20000, 256), ("c3", 40008, 64)])
-def test_reduced_tables(name, V, H):
-    _run(synth.WORKLOADS[name], [1.0, 0.5, 2.0], H=H, V=V)
+def test_reduced_tables(request, name, V, H):
+    _run(synth.WORKLOADS[name], [1.0, 0.5, 2.0], H=H, V=V, test_id=request.node.nodeid)
 
 
 @pytest.mark.parametrize("n,k,D,B,V", [(1, 4, 5, 3, 512), (6, 1, 6, 3, 512), (5, 8, 3, 4, 8), (7, 3, 4, 2, 12), (64, 10, 10, 2, 4099)])
-def test_edge_sizes(n, k, D, B, V):
-    _run(synth.Workload("edge", B, V, n, k, D, 3.0, 1.1, 0.3, H=64, seed=n * 1000 + k), [1.0, 0.3])
+def test_edge_sizes(request, n, k, D, B, V):
+    _run(synth.Workload("edge", B, V, n, k, D, 3.0, 1.1, 0.3, H=64, seed=n * 1000 + k), [1.0, 0.3], test_id=request.node.nodeid)
 
 
-def test_full_size_c4():
-    _run(synth.WORKLOADS["c4"], [1.0], steps=1)
+def test_full_size_c4(request):
+    _run(synth.WORKLOADS["c4"], [1.0], steps=1, test_id=request.node.nodeid)
 
 
 def test_low_temperature_is_the_greedy_walk():
