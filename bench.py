@@ -8,10 +8,13 @@ max depth 10 ("c4"), threshold off (every layer drafted, so the byte count is fi
 
   python bench.py [--gpus N] [--steps K] [--warmup W]         # CUDA path, one JSON line
   python bench.py --impl reference ...                        # the CPU oracle, same metric
+  python bench.py --rows N                                    # the row step alone (its own roofline line)
+  python bench.py --table-rows H                              # the same workload on a table of H rows
+  python bench.py --study mal                                 # acceptance lengths of adaptive and fixed trees
 
-With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs its own batch
-with its own seeds and tables (weak scaling, no data-path collective); the time is the maximum
-over ranks.
+With N > 1 every rank (one per GPU; started by torch.distributed.run, or by this program itself
+when it was started as a single process) runs its own batch with its own seeds and tables (weak
+scaling, no data-path collective); the time is the maximum over ranks.
 """
 from __future__ import annotations
 
@@ -28,11 +31,13 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2406_17276_b200 import synth  # noqa: E402
+from paper_2406_17276_b200 import shard, synth  # noqa: E402
 
 METRIC = "opt_tree_builds_per_s"
 UNIT = "trees/s"
 NEG_INF = -math.inf
+MIN_TIMED_MS = 500.0          # the timed region is repeated in blocks of --steps until it has lasted this long
+BIG_TABLE_ROWS = 32768        # rows of the table that defeats L2 reuse (2.1 GB at V=32000, 17 times the L2)
 
 
 def _peaks():
@@ -43,10 +48,9 @@ def _peaks():
 
 
 # DRAM bytes of one build_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
-# capture, see profiles/), keyed by workload, with the digest of the kernel sources the counters
-# were taken on: a changed kernel reports no traffic.
+# capture, see profiles/), keyed by workload and table rows, with the digest of the kernel sources the
+# counters were taken on: a changed kernel reports no traffic.
 NCU_TRAFFIC = {
-    "c4": {"bytes": 600.1e6, "csrc_sha256": "6ae3b61f2b8ac64cafa7e6b91a996773f37410eea89561611d0ded1bbae73f33"},
 }
 
 
@@ -61,8 +65,8 @@ def _csrc_digest() -> str:
     return h.hexdigest()
 
 
-def _ncu_traffic(workload: str, delta: float):
-    rec = NCU_TRAFFIC.get(workload)
+def _ncu_traffic(workload: str, H: int, delta: float):
+    rec = NCU_TRAFFIC.get((workload, H))
     if rec is None or delta != NEG_INF or rec["csrc_sha256"] != _csrc_digest():
         return None
     return rec["bytes"]
@@ -119,82 +123,220 @@ def logical_rows(w, depth_reached):
     return rows
 
 
+def describe(w, H, delta):
+    return (f"{w.name}: batch {w.batch} per GPU, V={w.V}, n={w.n}, k={w.k}, max_depth={w.max_depth}, "
+            f"delta={'off' if delta == NEG_INF else delta}, H={H} bf16 tables "
+            f"(sigma {w.sigma}, Zipf s {w.zipf_s}, {int(w.disagree * 100)}% rows disagree)")
+
+
+class EventTimer:
+    """CUDA events on the current stream, with the interface shard.timed_job expects."""
+
+    def __init__(self):
+        import torch
+        self.e0, self.e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def start(self):
+        self.e0.record()
+
+    def stop(self):
+        self.e1.record()
+
+    def elapsed_ms(self):
+        return self.e0.elapsed_time(self.e1)
+
+
+class Stepper:
+    """Device buffers of one workload and its decoding step through the binding."""
+
+    def __init__(self, w, ld, lt, local, with_target=True):
+        import torch
+        from paper_2406_17276_b200 import binding
+        self.torch, self.w = torch, w
+        self.H = ld.shape[0]
+        self.d_ld = torch.from_numpy(ld.view(np.int16)).cuda()
+        self.d_lt = torch.from_numpy(lt.view(np.int16)).cuda() if with_target else None
+        B, D = w.batch, w.max_depth
+        self.ot = binding.OptTree(w.V, self.H, w.n, w.k, D, B, device=f"cuda:{local}")
+        self.roots0 = torch.from_numpy(synth.root_tokens(B, w.V, w.seed + 1)).cuda()
+        self.base = torch.zeros(B, dtype=torch.int32, device="cuda")
+        self.tree = self.ot.alloc_tree(B, trace=False)
+        self.mask = torch.empty((B, w.n, self.ot.W), dtype=torch.int64, device="cuda")
+        self.pos = torch.empty((B, w.n), dtype=torch.int32, device="cuda")
+        i32 = dict(dtype=torch.int32, device="cuda")
+        self.vout = [(torch.empty(B, **i32), torch.empty((B, D + 1), **i32), torch.empty((B, D), **i32), torch.empty(B, **i32))
+                     for _ in range(2)]
+        self.root = self.roots0
+        self.build_events = []
+
+    def step(self, i, delta, time_build=False):
+        torch, ot = self.torch, self.ot
+        if time_build:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            ot.build(self.d_ld, self.root, delta, self.tree)
+            b.record()
+            self.build_events.append((a, b))
+        else:
+            ot.build(self.d_ld, self.root, delta, self.tree)
+        ot.mask(self.tree, self.base, self.mask, self.pos)
+        o = self.vout[i & 1]
+        ot.verify(self.tree, self.d_lt, self.root, o)
+        self.root = o[3]                             # next_root feeds the next step
+
+    def build_ms(self):
+        ms = [a.elapsed_time(b) for a, b in self.build_events]
+        return sum(ms) / len(ms) if ms else None
+
+    def check(self, what):
+        st = self.ot.device_status()
+        if st != 0:
+            raise SystemExit(f"bench.py: device status {st} after {what}")
+
+
+def _sync():
+    import torch
+    torch.cuda.synchronize()
+
+
+def timed_blocks(s: Stepper, steps, warmup, delta, max_build_events=4000):
+    """Blocks of exactly `steps` timed steps (shard.timed_job: barrier + synchronize on both sides, the
+    slowest rank's time) until the timed region has lasted MIN_TIMED_MS.  Returns (trees/s of the whole
+    job, ms per step, blocks)."""
+    B = s.w.batch
+    total_units_rate_ms, blocks, tot_ms = 0.0, 0, 0.0
+    units = 0.0
+    w_left = warmup
+    while True:
+        value, ms = shard.timed_job(lambda i: s.step(i, delta, time_build=len(s.build_events) < max_build_events and i >= w_left),
+                                    steps, w_left, B, EventTimer(), _sync, device="cuda")
+        w_left = 0
+        units += value * ms * 1e-3
+        tot_ms += ms
+        blocks += 1
+        if tot_ms >= MIN_TIMED_MS or blocks * steps >= 200000:
+            break
+    return units / (tot_ms * 1e-3), tot_ms / (blocks * steps), blocks
+
+
+def quick_config(name, local, delta=NEG_INF):
+    """Device-resident steps of another configuration, timed for a fraction of a second."""
+    import torch
+    w = synth.WORKLOADS[name]
+    ld, lt = synth.make_tables(w)
+    s = Stepper(w, ld, lt, local)
+    del ld, lt
+    for i in range(3):
+        s.step(i, delta)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(); s.step(0, delta); e1.record(); torch.cuda.synchronize()
+    est = max(e0.elapsed_time(e1), 1e-3)
+    steps = int(min(2000, max(5, 300.0 / est)))
+    s.build_events = []
+    t = EventTimer()
+    t.start()
+    for i in range(steps):
+        s.step(i, delta, time_build=True)
+    t.stop(); torch.cuda.synchronize()
+    s.check(name)
+    ms = t.elapsed_ms() / steps
+    bms = s.build_ms()
+    rows = logical_rows(w, s.tree.depth_reached.cpu().numpy())
+    peak, _ = _peaks()
+    gbs = 2.0 * w.V * rows / (bms * 1e-3) / 1e9
+    out = {"workload": describe(w, w.H, delta), "steps": steps, "trees_per_s": w.batch / (ms * 1e-3), "ms_per_step": ms,
+           "build_ms": bms, "rows_per_build_call": rows, "algorithmic_gbs": gbs, "frac": gbs / peak,
+           "frac_of_nominal_8000": gbs / 8000.0}
+    if w.batch == 1:
+        out["latency_ms_one_sequence"] = ms
+    del s
+    torch.cuda.empty_cache()
+    return out
+
+
+def big_table_build(w, local, H, delta=NEG_INF, calls=40):
+    """opt_tree_build alone on the same shape with a draft table of H rows: every row a build reads is then
+    a row the L2 does not hold, so the algorithmic bytes are bytes from HBM."""
+    import torch
+    from paper_2406_17276_b200 import binding
+    ld = synth.draft_table(w.V, w.sigma, w.zipf_s, w.seed, H)
+    d_ld = torch.from_numpy(ld.view(np.int16)).cuda()
+    del ld
+    ot = binding.OptTree(w.V, H, w.n, w.k, w.max_depth, w.batch, device=f"cuda:{local}")
+    roots = [torch.from_numpy(synth.root_tokens(w.batch, w.V, w.seed + 100 + i)).cuda() for i in range(8)]
+    tree = ot.alloc_tree(w.batch, trace=False)
+    for i in range(5):
+        ot.build(d_ld, roots[i % 8], delta, tree)
+    t = EventTimer()
+    torch.cuda.synchronize()
+    t.start()
+    for i in range(calls):
+        ot.build(d_ld, roots[i % 8], delta, tree)
+    t.stop(); torch.cuda.synchronize()
+    if ot.device_status() != 0:
+        raise SystemExit("bench.py: device status after the big-table builds")
+    ms = t.elapsed_ms() / calls
+    rows = logical_rows(w, tree.depth_reached.cpu().numpy())
+    peak, kind = _peaks()
+    gbs = 2.0 * w.V * rows / (ms * 1e-3) / 1e9
+    traffic = _ncu_traffic(w.name, H, delta)
+    out = {"table_rows": H, "table_bytes": 2.0 * w.V * H, "build_ms": ms, "calls": calls, "achieved": gbs, "unit": "GB/s",
+           "frac": gbs / peak, "peak_kind": f"of {kind}", "frac_of_nominal_8000": gbs / 8000.0, "traffic": traffic,
+           "frac_dram": (traffic / (ms * 1e-3) / 1e9 / peak) if traffic else None,
+           "note": "opt_tree_build alone, back to back, roots changing from call to call"}
+    del ot, d_ld
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_cuda(args):
     import torch
-    from paper_2406_17276_b200 import binding, build, shard
 
-    rank = int(os.environ.get("RANK", 0)); world = int(os.environ.get("WORLD_SIZE", 1))
-    local = int(os.environ.get("LOCAL_RANK", 0))
+    if args.gpus > 1 and not shard.launched_by_torchrun():
+        # asked for several GPUs as a single process: become the launcher of one rank per GPU
+        raise SystemExit(shard.launch_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    local = int(os.environ.get("LOCAL_RANK", 0))
     torch.cuda.set_device(local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    rank, world, local = shard.init_ranks("nccl", torch.device("cuda", local))
+    from paper_2406_17276_b200 import build
     build.build()
     w = shard.rank_workload(synth.WORKLOADS[args.workload], rank)
-    ld, lt = synth.make_tables(w)
-    d_ld = torch.from_numpy(ld.view(np.int16)).cuda(); d_lt = torch.from_numpy(lt.view(np.int16)).cuda()
-    B, D = w.batch, w.max_depth
-    ot = binding.OptTree(w.V, w.H, w.n, w.k, D, B, device=f"cuda:{local}")
-    roots0 = torch.from_numpy(synth.root_tokens(B, w.V, w.seed + 1)).cuda()
-    base = torch.zeros(B, dtype=torch.int32, device="cuda")
-    tree = ot.alloc_tree(B, trace=False)
-    mask = torch.empty((B, w.n, ot.W), dtype=torch.int64, device="cuda")
-    pos = torch.empty((B, w.n), dtype=torch.int32, device="cuda")
-    i32 = dict(dtype=torch.int32, device="cuda")
-    vout = [(torch.empty(B, **i32), torch.empty((B, D + 1), **i32), torch.empty((B, D), **i32), torch.empty(B, **i32))
-            for _ in range(2)]
-    delta = args.delta
+    H = args.table_rows or w.H
+    ld, lt = synth.make_tables(w, H=H)
+    s = Stepper(w, ld, lt, local)
+    ot, B, D, delta = s.ot, w.batch, w.max_depth, args.delta
+    warmup = max(3, args.warmup)
 
-    def step(i, root):
-        ot.build(d_ld, root, delta, tree)
-        ot.mask(tree, base, mask, pos)
-        o = vout[i & 1]
-        ot.verify(tree, d_lt, root, o)
-        return o[3]                                  # next_root feeds the next step
+    # one step from the first roots, kept for the comparison with the oracle in the cpu_baseline leg
+    s.step(0, delta)
+    torch.cuda.synchronize()
+    first = {f: getattr(s.tree, f).cpu().numpy() for f in ("token", "parent", "depth", "n_sel", "depth_reached")}
+    first.update(mask=s.mask.cpu().numpy().view(np.uint64), position_ids=s.pos.cpu().numpy(),
+                 accept_len=s.vout[0][0].cpu().numpy(), accept_tokens=s.vout[0][1].cpu().numpy(),
+                 accept_nodes=s.vout[0][2].cpu().numpy(), next_root=s.vout[0][3].cpu().numpy(),
+                 phat=s.tree.phat.cpu().numpy(), expected_len=s.tree.expected_len.cpu().numpy())
+    s.root = s.roots0
+
+    # ---- device-resident timing ----
+    sampler = ClockSampler(local); sampler.start()
+    launches0 = ot.launch_count()
+    value, ms_per_step, blocks = timed_blocks(s, args.steps, warmup, delta)
+    clocks = sampler.result()
+    launches = (ot.launch_count() - launches0) * args.steps // (blocks * args.steps + warmup)   # of one block of --steps
+    build_ms = s.build_ms()
+    s.check("the timed steps")
+    rows_total = logical_rows(w, s.tree.depth_reached.cpu().numpy())    # the last build's own count (all equal with the threshold off)
+    algo_bytes = 2.0 * w.V * rows_total
+    tree, mask, vout, d_ld, d_lt, roots0 = s.tree, s.mask, s.vout, s.d_ld, s.d_lt, s.roots0
 
     def barrier():
         if world > 1:
+            import torch.distributed as dist
             dist.barrier()
         torch.cuda.synchronize()
-
-    # ---- device-resident timing ----
-    root = roots0
-    for i in range(args.warmup):
-        root = step(i, root)
-    barrier()
-    sampler = ClockSampler(local); sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    bev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    rows_total = 0
-    launches0 = ot.launch_count()
-    ev0.record()
-    for i in range(args.steps):
-        bev[i][0].record()
-        ot.build(d_ld, root, delta, tree)
-        bev[i][1].record()
-        ot.mask(tree, base, mask, pos)
-        o = vout[i & 1]
-        ot.verify(tree, d_lt, root, o)
-        root = o[3]
-    ev1.record()
-    barrier()
-    clocks = sampler.result()
-    launches = ot.launch_count() - launches0
-    ms = ev0.elapsed_time(ev1)
-    build_ms = sum(a.elapsed_time(b) for a, b in bev) / args.steps
-    status = ot.device_status()
-    if status != 0:
-        raise SystemExit(f"bench.py: device status {status}")
-    # bytes of the last build (all builds are identical in size when the threshold is off)
-    rows_last = logical_rows(w, tree.depth_reached.cpu().numpy())
-    if delta == NEG_INF:
-        rows_total = rows_last
-    else:
-        rows_total = rows_last            # threshold on: the last build's own count is reported
-    algo_bytes = 2.0 * w.V * rows_total
-    value, ms = shard.whole_job(B * args.steps, ms, device="cuda")       # all ranks' trees / the slowest rank's time
 
     # ---- end to end through the host-buffer entry point ----
     ho = ot.alloc_host_out(B)
@@ -217,120 +359,128 @@ def run_cuda(args):
     h2d = 2 * B * 4
     d2h = sum(int(t.numel() * t.element_size()) for t in ho.values())
 
-    # ---- the bookkeeping after verification (dense mask, cache keep list): timed on its own, not part of a step ----
+    peak, peak_kind = _peaks()
+    achieved = algo_bytes / (build_ms * 1e-3) / 1e9
+    traffic = args.traffic if args.traffic is not None else _ncu_traffic(args.workload, H, args.delta)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": describe(w, H, delta),
+                   "l2": f"inputs larger than L2: two {2.0 * w.V * H / 1e6:.0f} MB tables against a 126 MB L2, no explicit flush",
+                   "step": "build + mask + verify, next roots from verify",
+                   "timed_region": f"{blocks} blocks of {args.steps} steps (repeated until {MIN_TIMED_MS:.0f} ms), "
+                                   "each block between barriers; value and ms_per_step are over all blocks"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "build_kernel (opt_tree_build: one persistent kernel per call)",
+                     "achieved": achieved, "achieved_kind": "algorithmic bytes (rows read once each; with 4096 table rows part of them is served by L2)",
+                     "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / 8000.0,
+                     "algorithmic_bytes_per_build_call": algo_bytes, "build_ms": build_ms,
+                     "traffic": traffic,
+                     "frac_dram": (traffic / (build_ms * 1e-3) / 1e9 / peak) if traffic else None},
+    }
+    if world == 1 and not args.quick:
+        line.update(extras(s, args, local, rows_total))
+    del s
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            cb, o_first = cpu_baseline(w, ld, lt, steps=2, want_first=True)
+            line["cpu_baseline"] = cb
+            line["cpu_baseline_all_cores"] = cpu_baseline_all_cores(w, ld, lt)
+            line["parity"] = parity_counts(first, o_first)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    if rank == 0 and line.get("parity", {}).get("mismatch", 0):
+        raise SystemExit("bench.py: the checked step differs from the oracle beyond the near-tie rule")
+
+
+def extras(s: Stepper, args, local, rows_total):
+    """Entry points outside the timed step, each timed alone, the same workload on a table that defeats L2
+    reuse, and the other configurations (one GPU only)."""
+    import torch
+    ot, w, tree, mask, vout, d_ld, d_lt, roots0 = s.ot, s.w, s.tree, s.mask, s.vout, s.d_ld, s.d_lt, s.roots0
+    B, D, delta = w.batch, w.max_depth, args.delta
+    i32 = dict(dtype=torch.int32, device="cuda")
+    out = {}
+
+    def timed(fn, reps, warm=3):
+        for _ in range(warm):
+            fn(0)
+        t = EventTimer()
+        torch.cuda.synchronize()
+        t.start()
+        for i in range(reps):
+            fn(i)
+        t.stop(); torch.cuda.synchronize()
+        return t.elapsed_ms() / reps
+
+    # bookkeeping after verification (dense mask, cache keep list)
     pv_out = ot.post_verify(tree, mask, vout[0][0], vout[0][2])
-    for _ in range(5):
-        ot.post_verify(tree, mask, vout[0][0], vout[0][2], pv_out)
-    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    p0.record()
-    for _ in range(100):
-        ot.post_verify(tree, mask, vout[0][0], vout[0][2], pv_out)
-    p1.record(); torch.cuda.synchronize()
-    post_verify_us = p0.elapsed_time(p1) * 10.0
-    if ot.device_status() != 0:
-        raise SystemExit("bench.py: device status after post_verify")
+    pv_ms = timed(lambda i: ot.post_verify(tree, mask, vout[0][0], vout[0][2], pv_out), 100, 5)
+    s.check("post_verify")
+    out["post_verify"] = {"us_per_call": pv_ms * 1e3, "bytes_written": int(sum(t.numel() * t.element_size() for t in pv_out)),
+                          "note": "opt_tree_post_verify alone, back-to-back calls; not part of the timed step"}
 
-    # ---- the pruned draft (same trees from fewer rows): timed on its own, with its own byte count ----
-    rows_read = torch.empty(B, dtype=torch.int32, device="cuda")
-    for _ in range(5):
-        ot.build_pruned(d_ld, roots0, delta, tree, rows_read)
-    q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    q0.record()
-    for _ in range(50):
-        ot.build_pruned(d_ld, roots0, delta, tree, rows_read)
-    q1.record(); torch.cuda.synchronize()
-    pruned_ms = q0.elapsed_time(q1) / 50
+    # the pruned draft (same trees from fewer rows)
+    rows_read = torch.empty(B, **i32)
+    pruned_ms = timed(lambda i: ot.build_pruned(d_ld, roots0, delta, tree, rows_read), 50, 5)
     pruned_rows = int(rows_read.sum().item())
-    if ot.device_status() != 0:
-        raise SystemExit("bench.py: device status after build_pruned")
+    s.check("build_pruned")
+    out["pruned_build"] = {"ms_per_build": pruned_ms, "trees_per_s": B / (pruned_ms * 1e-3), "rows_read": pruned_rows,
+                           "rows_of_full_build": int(rows_total), "gbs_of_rows_read": 2.0 * w.V * pruned_rows / (pruned_ms * 1e-3) / 1e9,
+                           "note": "opt_tree_build_pruned alone on the first step's roots: the same trees, only rows that can still matter; not the benchmark's metric"}
 
-    # ---- the layer-by-layer build (logits handed in per layer, as a real draft model would): timed on its own.
-    #      The table plays the model; every layer's logits are gathered beforehand, only the library's calls are timed.
+    # the layer-by-layer build: the table plays the model; every layer's logits are gathered beforehand
     layers_ms, layer_bufs = None, []
-    if 2.0 * w.V * B * (1 + (D - 1) * w.n) <= 4e9:          # the pre-gathered logits of all layers must fit comfortably
+    if 2.0 * w.V * B * (1 + (D - 1) * w.n) <= 4e9:
         ot.layers_begin(B)
         ltoks = roots0.view(-1, 1).to(torch.int64)
-        lcnt = torch.ones(B, dtype=torch.int32, device="cuda")
+        lcnt = torch.ones(B, **i32)
         for depth in range(D):
             stride = int(lcnt.max().item())
             if stride == 0:
                 break
-            lrows = (ltoks[:, :stride] * 31 + depth) % w.H
+            lrows = (ltoks[:, :stride] * 31 + depth) % s.H
             layer_bufs.append(d_ld[lrows.reshape(-1)].reshape(B, stride, w.V).contiguous())
             nt, _, lcnt = ot.layers_step(layer_bufs[-1], delta, tree)
             ltoks = nt.to(torch.int64)
         lnxt = (torch.empty((B, w.n), **i32), torch.empty((B, w.n), **i32), torch.empty(B, **i32))
 
-        def layers_run():
+        def layers_run(_i):
             ot.layers_begin(B)
             for lg in layer_bufs:
                 ot.layers_step(lg, delta, tree, lnxt)
 
-        for _ in range(3):
-            layers_run()
-        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        l0.record()
-        for _ in range(20):
-            layers_run()
-        l1.record(); torch.cuda.synchronize()
-        layers_ms = l0.elapsed_time(l1) / 20
-        if ot.device_status() != 0:
-            raise SystemExit("bench.py: device status after layers_step")
+        layers_ms = timed(layers_run, 20)
+        s.check("layers_step")
         del layer_bufs[:]
+    out["layers_build"] = {"ms_per_batch": layers_ms, "trees_per_s": (B / (layers_ms * 1e-3)) if layers_ms else None,
+                           "note": "opt_tree_layers_begin + one opt_tree_layers_step per layer on pre-gathered logits; not the benchmark's metric"}
 
-    # ---- verification with sampling (temperature 1): timed on its own ----
+    # verification with sampling (temperature 1)
+    ot.build(d_ld, roots0, delta, tree)
     sv_out = ot.verify_sampled(tree, d_lt, roots0, 1.0, 2024, 0)
-    for _ in range(3):
-        ot.verify_sampled(tree, d_lt, roots0, 1.0, 2024, 0, sv_out)
-    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    s0.record()
-    for i in range(50):
-        ot.verify_sampled(tree, d_lt, roots0, 1.0, 2024, i, sv_out)
-    s1.record(); torch.cuda.synchronize()
-    verify_sampled_us = s0.elapsed_time(s1) * 20.0
-    if ot.device_status() != 0:
-        raise SystemExit("bench.py: device status after verify_sampled")
+    sv_ms = timed(lambda i: ot.verify_sampled(tree, d_lt, roots0, 1.0, 2024, i, sv_out), 50)
+    s.check("verify_sampled")
+    sv_rows = int(tree.n_sel.sum().item()) + B
+    out["verify_sampled"] = {"us_per_call": sv_ms * 1e3, "target_rows": sv_rows,
+                             "algorithmic_gbs": 2.0 * w.V * sv_rows / (sv_ms * 1e-3) / 1e9,
+                             "note": "opt_tree_verify_sampled alone at temperature 1; not part of the timed step"}
+    gv_ms = timed(lambda i: ot.verify(tree, d_lt, roots0, vout[0]), 50)
+    out["verify_greedy"] = {"us_per_call": gv_ms * 1e3, "target_rows": sv_rows,
+                            "algorithmic_gbs": 2.0 * w.V * sv_rows / (gv_ms * 1e-3) / 1e9}
 
-    peak, peak_kind = _peaks()
-    achieved = algo_bytes / (build_ms * 1e-3) / 1e9
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{w.name}: batch {B} per GPU, V={w.V}, n={w.n}, k={w.k}, max_depth={D}, "
-                               f"delta={'off' if delta == NEG_INF else delta}, H={w.H} bf16 tables "
-                               f"(sigma {w.sigma}, Zipf s {w.zipf_s}, {int(w.disagree * 100)}% rows disagree)",
-                   "l2": "inputs larger than L2: two 262 MB tables against a 126 MB L2, no explicit flush",
-                   "step": "build + mask + verify, next roots from verify"},
-        "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": int(launches),
-        "pruned_build": {"ms_per_build": pruned_ms, "trees_per_s": B / (pruned_ms * 1e-3), "rows_read": pruned_rows,
-                         "rows_of_full_build": int(rows_total), "gbs_of_rows_read": 2.0 * w.V * pruned_rows / (pruned_ms * 1e-3) / 1e9,
-                         "note": "opt_tree_build_pruned alone on the first step's roots: the same trees, only rows that can still matter; not the benchmark's metric"},
-        "layers_build": {"ms_per_batch": layers_ms, "trees_per_s": (B / (layers_ms * 1e-3)) if layers_ms else None,
-                         "note": "opt_tree_layers_begin + one opt_tree_layers_step per layer on pre-gathered logits (two launches per layer; skipped when those logits would not fit); not the benchmark's metric"},
-        "verify_sampled": {"us_per_call": verify_sampled_us,
-                           "note": "opt_tree_verify_sampled alone at temperature 1 (one double-precision exponential per target logit); not part of the timed step"},
-        "post_verify": {"us_per_call": post_verify_us, "bytes_written": int(sum(t.numel() * t.element_size() for t in pv_out)),
-                        "note": "opt_tree_post_verify alone, 100 back-to-back calls; not part of the timed step"},
-        "roofline": {"bound": "hbm", "kernel": "build_kernel (opt_tree_build: init_build_kernel + one persistent build_kernel)",
-                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / 8000.0,
-                     "algorithmic_bytes_per_build_call": algo_bytes, "build_ms": build_ms,
-                     "traffic": args.traffic if args.traffic is not None else _ncu_traffic(args.workload, args.delta)},
-    }
-    if rank == 0:
-        if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(w, ld, lt, steps=2)
-        print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    if args.table_rows == 0 and args.workload == "c4":
+        out["big_table"] = big_table_build(w, local, BIG_TABLE_ROWS, delta)
+    if args.workload == "c4" and args.table_rows == 0 and not args.no_other_configs:
+        out["other_configs"] = {name: quick_config(name, local) for name in ("c1", "c2", "c3", "c5")}
+    return out
 
 
 def run_rows(args):
@@ -343,11 +493,12 @@ def run_rows(args):
         raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
     build.build()
     w = synth.WORKLOADS[args.workload]
-    ld, _ = synth.make_tables(w)
+    H = args.table_rows or w.H
+    ld = synth.draft_table(w.V, w.sigma, w.zipf_s, w.seed, H)
     d_ld = torch.from_numpy(ld.view(np.int16)).cuda()
-    ot = binding.OptTree(w.V, w.H, w.n, w.k, w.max_depth, w.batch)
+    ot = binding.OptTree(w.V, H, w.n, w.k, w.max_depth, w.batch)
     nrows = args.rows
-    rows = torch.from_numpy(np.random.default_rng(w.seed).integers(0, w.H, nrows).astype(np.int32)).cuda()
+    rows = torch.from_numpy(np.random.default_rng(w.seed).integers(0, H, nrows).astype(np.int32)).cuda()
     for _ in range(max(3, args.warmup)):
         ot.row_softmax_topk(d_ld, rows)
     torch.cuda.synchronize()
@@ -367,26 +518,76 @@ def run_rows(args):
     print(json.dumps({
         "metric": "rows_per_s", "value": nrows / (ms * 1e-3), "unit": "rows/s", "n_gpus": 1, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{w.name}: row step alone, {nrows} random rows of V={w.V}, k={w.k}, H={w.H} bf16 table",
-                   "l2": "the 262 MB table is larger than L2; rows repeat across the list"},
+        "config": {"workload": f"{w.name}: row step alone, {nrows} random rows of V={w.V}, k={w.k}, H={H} bf16 table",
+                   "l2": f"the {2.0 * w.V * H / 1e6:.0f} MB table is larger than L2; rows repeat across the list"},
         "clocks": clocks, "gpu_launches": args.steps,
         "roofline": {"bound": "hbm", "kernel": "row_topk_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": algo, "traffic": None},
     }), flush=True)
 
 
-def cpu_baseline(w, ld, lt, steps, batch=None):
+def cpu_baseline(w, ld, lt, steps, batch=None, want_first=False):
     """The oracle as it stands, single thread, un-memoised, on a bounded sample of the workload."""
     import oracle
     B = batch or w.batch
     roots = synth.root_tokens(B, w.V, w.seed + 1)
+    first = None
     t0 = time.perf_counter()
     for _ in range(steps):
         r = oracle.table_step(ld, lt, roots, w.n, w.k, w.max_depth, NEG_INF)
+        first = first or r
         roots = r.next_root.copy()
     dt = time.perf_counter() - t0
-    return {"value": B * steps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"{steps} steps of {B} sequences (build + mask + verify), threshold off, no memo", "seconds": dt}
+    cb = {"value": B * steps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+          "sample": f"{steps} steps of {B} sequences (build + mask + verify), threshold off, no memo", "seconds": dt}
+    return (cb, first) if want_first else cb
+
+
+def cpu_baseline_all_cores(w, ld, lt, per_thread=2):
+    """The same oracle code on every host core: one thread per core, each taking sequences of its own
+    (the C routine runs without the interpreter lock)."""
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+    P = os.cpu_count() or 1
+    roots = synth.root_tokens(P * per_thread, w.V, w.seed + 2)
+    oracle.lib()
+
+    def work(t):
+        for j in range(per_thread):
+            oracle.table_step(ld, lt, roots[t * per_thread + j:t * per_thread + j + 1], w.n, w.k, w.max_depth, NEG_INF)
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(P) as ex:
+        list(ex.map(work, range(P)))
+    dt = time.perf_counter() - t0
+    return {"value": P * per_thread / dt, "unit": UNIT, "cores": P, "kind": "oracle",
+            "sample": f"{per_thread} sequences on each of {P} threads (build + mask + verify), threshold off, no memo", "seconds": dt}
+
+
+def parity_counts(g, o):
+    """The checked step (the first roots, threshold off) against the oracle's result for it: sequences whose
+    integer outputs are identical; sequences that differ where the oracle reports a selection boundary closer
+    than 1e-6 relative (near ties); anything else is a mismatch.  Largest relative errors of the path values
+    and of E(A) over the identical ones."""
+    B = g["n_sel"].shape[0]
+    out = dict(exact=0, near_tie=0, stop_near_tie=0, mismatch=0, max_phat_rel=0.0, max_elen_rel=0.0, sequences=B)
+    ints = ("token", "parent", "depth", "n_sel", "depth_reached", "mask", "position_ids", "accept_len", "accept_tokens",
+            "accept_nodes", "next_root")
+    for b in range(B):
+        if all(np.array_equal(np.asarray(g[f][b]), np.asarray(getattr(o, f)[b])) for f in ints):
+            out["exact"] += 1
+            ns = int(o.n_sel[b])
+            rel = float(np.max(np.abs(g["phat"][b, :ns] - o.phat[b, :ns]) / o.phat[b, :ns])) if ns else 0.0
+            er = float(abs(g["expected_len"][b] - o.expected_len[b]) / o.expected_len[b])
+            out["max_phat_rel"] = max(out["max_phat_rel"], rel)
+            out["max_elen_rel"] = max(out["max_elen_rel"], er)
+            if rel > 1e-5 or er > 1e-5:
+                out["mismatch"] += 1
+        elif o.min_gap[b] < 1e-6:
+            out["near_tie"] += 1
+        else:
+            out["mismatch"] += 1
+    return out
 
 
 def run_reference(args):
@@ -397,7 +598,7 @@ def run_reference(args):
     oracle.build()
     w = synth.WORKLOADS[args.workload]
     ld, lt = synth.make_tables(w)
-    sample_b = 8                                        # bounded sample per step: 8 of the 32 sequences
+    sample_b = min(8, w.batch)                          # bounded sample per step: 8 of the batch's sequences
     steps, warm = max(1, min(args.steps, 4)), max(0, min(args.warmup, 1))
     if warm:
         cpu_baseline(w, ld, lt, warm, batch=sample_b)
@@ -421,13 +622,24 @@ def main():
     ap.add_argument("--workload", default="c4", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--delta", type=float, default=NEG_INF)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the other four configurations")
+    ap.add_argument("--quick", action="store_true", help="only the timed steps and the end-to-end leg")
+    ap.add_argument("--table-rows", type=int, default=0,
+                    help="rows H of the logit tables (default: the workload's 4096); e.g. 32768 makes every row a build reads come from HBM")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu dram bytes per build call to report in roofline.traffic (default: the recorded capture, if the kernel sources are unchanged)")
     ap.add_argument("--rows", type=int, default=0,
                     help="time the row step alone over this many rows instead of whole steps (its own roofline line)")
+    ap.add_argument("--study", default=None, choices=["mal"],
+                    help="mal: mean acceptance length and E(A) of OPT-Tree against fixed trees of the same size on the synthetic tables")
     args = ap.parse_args()
     if args.impl == "reference":
+        if args.gpus > 1 and not shard.launched_by_torchrun():
+            raise SystemExit(shard.launch_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
         run_reference(args)
+    elif args.study:
+        from paper_2406_17276_b200 import study
+        study.main(args)
     elif args.rows > 0:
         run_rows(args)
     else:

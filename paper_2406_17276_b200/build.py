@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libopt_tree.so")
 SOURCES = [os.path.join(CSRC, "opt_tree.cu")]
-NVCC_FLAGS = os.environ.get("OT_EXTRA_NVCC", "").split() + ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-maxrregcount=80",
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-maxrregcount=80",
               "-shared", "-Xcompiler", "-fPIC"]
 
 
@@ -23,7 +23,7 @@ def _stale() -> bool:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
-        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+        nvcc = "/usr/local/cuda/bin/nvcc"
         cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + SOURCES
         subprocess.check_call(cmd)
     return LIB

@@ -65,3 +65,34 @@ def test_rank_workload_keeps_the_shape():
 
 def test_single_process_needs_no_group():
     assert shard.whole_job(8.0, 4.0) == (2000.0, 4.0)
+
+
+@pytest.mark.timeout(300)
+def test_launcher_starts_one_rank_per_gpu_and_the_job_is_timed_over_all_of_them(tmp_path):
+    """shard.launch_ranks + shard.timed_job with gloo ranks and a stand-in step: the job's time is the
+    slow rank's, its units are both ranks'."""
+    import json
+    import sys
+    out = tmp_path / "line.json"
+    stub = os.path.join(os.path.dirname(os.path.abspath(__file__)), "_stub_ranks.py")
+    rc = shard.launch_ranks(stub, [str(out), "10"], 2)
+    assert rc == 0
+    line = json.load(open(out))
+    assert line["n_gpus"] == 2 and line["calls"] == 12            # 2 warm-up + 10 timed steps on rank 0
+    assert line["ms"] >= 10 * 4.0 * 0.9                           # rank 1 sleeps 4 ms per step
+    assert line["value"] == pytest.approx(2 * 4.0 * 10 / (line["ms"] * 1e-3))
+
+
+@pytest.mark.timeout(300)
+def test_bench_asked_for_two_gpus_starts_two_ranks_by_itself():
+    """Without a CUDA device both ranks must stop at the "no CUDA device" exit: the CUDA path has no fallback."""
+    import subprocess
+    import sys
+    bench = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "bench.py")
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    if torch.cuda.is_available():
+        pytest.skip("needs a machine without a CUDA device")
+    p = subprocess.run([sys.executable, bench, "--gpus", "2", "--steps", "1", "--warmup", "0"], env=env,
+                       capture_output=True, text=True)
+    assert p.returncode != 0
+    assert (p.stdout + p.stderr).count("no CUDA device") == 2
