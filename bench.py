@@ -297,7 +297,8 @@ def run_cuda(args):
         # asked for several GPUs as a single process: become the launcher of one rank per GPU
         raise SystemExit(shard.launch_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
     if not torch.cuda.is_available():
-        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+        raise SystemExit(f"bench.py: rank {os.environ.get('RANK', 0)} of {os.environ.get('WORLD_SIZE', 1)}: "
+                         "no CUDA device (the CUDA path has no CPU fallback)")
     local = int(os.environ.get("LOCAL_RANK", 0))
     torch.cuda.set_device(local)
     rank, world, local = shard.init_ranks("nccl", torch.device("cuda", local))

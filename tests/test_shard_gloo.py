@@ -85,7 +85,8 @@ def test_launcher_starts_one_rank_per_gpu_and_the_job_is_timed_over_all_of_them(
 
 @pytest.mark.timeout(300)
 def test_bench_asked_for_two_gpus_starts_two_ranks_by_itself():
-    """Without a CUDA device both ranks must stop at the "no CUDA device" exit: the CUDA path has no fallback."""
+    """Without a CUDA device the ranks must stop at the "no CUDA device" exit (the CUDA path has no fallback);
+    the launcher ends the other rank as soon as the first has failed, so one message is certain, two are not."""
     import subprocess
     import sys
     bench = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "bench.py")
@@ -95,4 +96,5 @@ def test_bench_asked_for_two_gpus_starts_two_ranks_by_itself():
     p = subprocess.run([sys.executable, bench, "--gpus", "2", "--steps", "1", "--warmup", "0"], env=env,
                        capture_output=True, text=True)
     assert p.returncode != 0
-    assert (p.stdout + p.stderr).count("no CUDA device") == 2
+    text = p.stdout + p.stderr
+    assert "of 2: no CUDA device" in text                          # a rank of a two-rank job said so
