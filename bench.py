@@ -199,12 +199,12 @@ def _sync():
     torch.cuda.synchronize()
 
 
-def timed_blocks(s: Stepper, steps, warmup, delta, max_build_events=4000):
+def timed_blocks(s: Stepper, steps, warmup, delta, min_ms=MIN_TIMED_MS, max_build_events=4000):
     """Blocks of exactly `steps` timed steps (shard.timed_job: barrier + synchronize on both sides, the
     slowest rank's time) until the timed region has lasted MIN_TIMED_MS.  Returns (trees/s of the whole
     job, ms per step, blocks)."""
     B = s.w.batch
-    total_units_rate_ms, blocks, tot_ms = 0.0, 0, 0.0
+    blocks, tot_ms = 0, 0.0
     units = 0.0
     w_left = warmup
     while True:
@@ -214,7 +214,7 @@ def timed_blocks(s: Stepper, steps, warmup, delta, max_build_events=4000):
         units += value * ms * 1e-3
         tot_ms += ms
         blocks += 1
-        if tot_ms >= MIN_TIMED_MS or blocks * steps >= 200000:
+        if tot_ms >= min_ms or blocks * steps >= 200000:
             break
     return units / (tot_ms * 1e-3), tot_ms / (blocks * steps), blocks
 
@@ -324,7 +324,7 @@ def run_cuda(args):
     # ---- device-resident timing ----
     sampler = ClockSampler(local); sampler.start()
     launches0 = ot.launch_count()
-    value, ms_per_step, blocks = timed_blocks(s, args.steps, warmup, delta)
+    value, ms_per_step, blocks = timed_blocks(s, args.steps, warmup, delta, args.min_timed_ms)
     clocks = sampler.result()
     launches = (ot.launch_count() - launches0) * args.steps // (blocks * args.steps + warmup)   # of one block of --steps
     build_ms = s.build_ms()
@@ -370,7 +370,7 @@ def run_cuda(args):
         "config": {"workload": describe(w, H, delta),
                    "l2": f"inputs larger than L2: two {2.0 * w.V * H / 1e6:.0f} MB tables against a 126 MB L2, no explicit flush",
                    "step": "build + mask + verify, next roots from verify",
-                   "timed_region": f"{blocks} blocks of {args.steps} steps (repeated until {MIN_TIMED_MS:.0f} ms), "
+                   "timed_region": f"{blocks} blocks of {args.steps} steps (repeated until {args.min_timed_ms:.0f} ms), "
                                    "each block between barriers; value and ms_per_step are over all blocks"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -624,6 +624,8 @@ def main():
     ap.add_argument("--delta", type=float, default=NEG_INF)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-configs", action="store_true", help="skip the other four configurations")
+    ap.add_argument("--min-timed-ms", type=float, default=MIN_TIMED_MS,
+                    help="repeat the block of --steps timed steps until the timed region has lasted this long (0: one block, for profiler runs)")
     ap.add_argument("--quick", action="store_true", help="only the timed steps and the end-to-end leg")
     ap.add_argument("--table-rows", type=int, default=0,
                     help="rows H of the logit tables (default: the workload's 4096); e.g. 32768 makes every row a build reads come from HBM")

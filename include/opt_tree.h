@@ -242,6 +242,19 @@ int opt_tree_step_host(opt_tree_ctx *ctx, const void *draft_logits_bf16, const v
                        const int32_t *root_token_host, const int32_t *base_pos_host, int32_t B, float delta,
                        const opt_tree_host_out *out, void *stream);
 
+/* Self-test of the library's bounded device-side waits (not a step of the paper's method; the
+ * persistent build waits on mailboxes, counters and shared-memory barriers, each wait with a limit
+ * after which it records OPT_TREE_ERR_TIMEOUT and returns instead of hanging).  Launches one small
+ * kernel in which each kind of wait is entered on something nobody completes, with a limit of
+ * about 2^16 clock cycles (or 2^10 polls): a shared-memory barrier awaited by a whole warp, one
+ * awaited by a single thread, a candidate path-value word, a candidate token word, and the row
+ * fetcher's mailbox poll loop.
+ *   result (dev) [OPT_TREE_SELFTEST_WAITS] int32: one status word per wait, in that order; each must
+ *                read OPT_TREE_ERR_TIMEOUT once the stream has been synchronised
+ * The context's own status word is not touched.  Enqueues two small memsets and the kernel. */
+#define OPT_TREE_SELFTEST_WAITS 5
+int opt_tree_selftest_waits(opt_tree_ctx *ctx, int32_t *result, void *stream);
+
 /* Reads (and clears) the device status word; synchronises the device.  *status_host is
  * OPT_TREE_OK or the first device-side error recorded since the last call. */
 int opt_tree_last_device_status(opt_tree_ctx *ctx, int32_t *status_host);

@@ -20,7 +20,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -
 EXPORTS = ["opt_tree_workspace_bytes", "opt_tree_create", "opt_tree_destroy", "opt_tree_build", "opt_tree_mask",
            "opt_tree_verify", "opt_tree_row_softmax_topk", "opt_tree_step_host", "opt_tree_last_device_status",
            "opt_tree_launch_count", "opt_tree_strerror", "opt_tree_verify_static", "opt_tree_post_verify", "opt_tree_build_pruned", "opt_tree_layers_begin",
-           "opt_tree_layers_step", "opt_tree_verify_sampled"]
+           "opt_tree_layers_step", "opt_tree_verify_sampled", "opt_tree_selftest_waits"]
 
 
 class Config(C.Structure):
@@ -75,6 +75,7 @@ def lib():
                                            C.c_void_p, C.c_void_p, C.c_void_p]
         L.opt_tree_post_verify.argtypes = [C.c_void_p, C.POINTER(Out), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.opt_tree_selftest_waits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.opt_tree_strerror.restype = C.c_char_p
         L.opt_tree_strerror.argtypes = [C.c_int]
         _lib = L
@@ -262,6 +263,12 @@ class OptTree:
         _check(lib().opt_tree_step_host(self._ctx, _ptr(draft), _ptr(target), _ptr(root_token_host), _ptr(base_pos_host),
                                         B, C.c_float(delta), C.byref(ho), _stream()), "opt_tree_step_host")
         return host_out
+
+    def selftest_waits(self) -> torch.Tensor:
+        """opt_tree_selftest_waits: one status word per kind of bounded wait (each should read ERR_TIMEOUT)."""
+        res = torch.full((5,), 77, dtype=torch.int32, device=self.device)
+        _check(lib().opt_tree_selftest_waits(self._ctx, _ptr(res), _stream()), "opt_tree_selftest_waits")
+        return res
 
     def device_status(self) -> int:
         st = C.c_int32(0)

@@ -40,8 +40,10 @@ __device__ __forceinline__ void set_status(int* status, int code) {
 
 // Every wait in the library is bounded by this many SM clock cycles (about two seconds); on
 // expiry the waiter records kErrTimeout in the status word and gives up, so a protocol error
-// ends as an error code, never as a hang.
+// ends as an error code, never as a hang.  The waits take the limit as an argument only so that
+// the self-test (opt_tree_selftest_waits) can make each of them run out within microseconds.
 constexpr long long kWaitCycles = 1ll << 32;
+constexpr int kWaitPolls = 1 << 22;                 // limit of the waits that count polls instead of cycles
 
 // ---------------------------------------------------------------------------------------------
 // bf16 bit pattern -> 16-bit key whose unsigned order equals the numeric order of the values
@@ -145,7 +147,7 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
 // Bounded wait, called by every lane of a converged warp (try_wait suspends the thread in hardware
 // for a while, so the loop turns over slowly; the clock is read only once in 256 turns).  Returns
 // false to the whole warp (status set) when kWaitCycles pass without completion.
-__device__ __forceinline__ bool mbar_wait_warp(unsigned long long* bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait_warp(unsigned long long* bar, uint32_t parity, int* status, long long limit = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     long long t0 = 0;
     int turns = 0;
@@ -154,7 +156,7 @@ __device__ __forceinline__ bool mbar_wait_warp(unsigned long long* bar, uint32_t
         if ((++turns & 255) == 0) {
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitCycles) { ok = false; break; }
+            else if (now - t0 > limit) { ok = false; break; }
         }
     }
     if (!ok) set_status(status, kErrTimeout);
@@ -171,7 +173,7 @@ __device__ __forceinline__ bool mbar_test_wait(unsigned long long* bar, uint32_t
     return ok != 0;
 }
 // The same wait for a single thread whose warp mates are busy elsewhere (no warp-wide vote).
-__device__ __forceinline__ bool mbar_wait_thread(unsigned long long* bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait_thread(unsigned long long* bar, uint32_t parity, int* status, long long limit = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     long long t0 = 0;
     int turns = 0;
@@ -179,7 +181,7 @@ __device__ __forceinline__ bool mbar_wait_thread(unsigned long long* bar, uint32
         if ((++turns & 255) == 0) {
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitCycles) { set_status(status, kErrTimeout); return false; }
+            else if (now - t0 > limit) { set_status(status, kErrTimeout); return false; }
         }
     }
     return true;

@@ -945,6 +945,37 @@ verify_sampled_kernel(Workspace w, Params p, const uint16_t* __restrict__ target
     verify_tail(s, w, p, b, j, ns, y, tok, par, accept_len, accept_tokens, accept_nodes, next_root);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Self-test of the bounded waits: one CTA whose warps each enter one kind of wait on something that
+// nobody will ever complete or write (a fresh mbarrier, words that stay zero, a source that never has
+// a row), with a limit of microseconds.  Every wait must give up, record kErrTimeout in its own
+// status word and let the kernel end.  No bulk copy is in flight and nothing else runs in the CTA.
+// ------------------------------------------------------------------------------------------------
+struct NeverSource {
+    static constexpr bool kHasEmpty = false;
+    __device__ long long claim(int i) { return i; }
+    __device__ int poll(long long, RowDesc&, bool) { return 0; }
+};
+__global__ void __launch_bounds__(kThreads)
+wait_probe_kernel(int* result, const unsigned long long* zero_words, long long limit, int polls) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
+    pipeline_init(s);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == 0) {
+        mbar_wait_warp(&s.full_bar[0], 0u, &result[0], limit);
+    } else if (warp == 1) {
+        if (lane == 0) mbar_wait_thread(&s.full_bar[1], 0u, &result[1], limit);
+    } else if (warp == 2) {
+        if (lane == 0) poll_phat_word(zero_words, &result[2], polls);
+    } else if (warp == 3) {
+        if (lane == 0) poll_tok_word(reinterpret_cast<const unsigned int*>(zero_words + 1), &result[3], polls);
+    } else if (warp == 4) {
+        NeverSource src;
+        fetcher_role(s, src, &result[4], limit);
+    }
+}
+
 }  // namespace ot
 
 // ------------------------------------------------------------------------------------------------
@@ -1236,6 +1267,21 @@ int opt_tree_step_host(opt_tree_ctx* ctx, const void* draft, const void* target,
     OT_OUT(ho->accept_nodes, w.o_anode, Bz * D * 4) OT_OUT(ho->next_root, w.o_next, Bz * 4)
 #undef OT_OUT
     return OPT_TREE_OK;
+}
+
+int opt_tree_selftest_waits(opt_tree_ctx* ctx, int32_t* result, void* stream) {
+    if (!ctx || !result) return OPT_TREE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaFuncSetAttribute(ot::wait_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
+        cudaMemsetAsync(result, 0, OPT_TREE_SELFTEST_WAITS * sizeof(int32_t), st) != cudaSuccess ||
+        cudaMemsetAsync(ctx->ws.rprob, 0, 2 * sizeof(unsigned long long), st) != cudaSuccess) {     // two words nobody writes
+        cudaGetLastError();
+        return OPT_TREE_ERR_CUDA;
+    }
+    ot::wait_probe_kernel<<<1, ot::kThreads, sizeof(ot::CtaSmem), st>>>(
+        result, reinterpret_cast<const unsigned long long*>(ctx->ws.rprob), 1ll << 16, 1 << 10);
+    ctx->launches++;
+    return check_launch();
 }
 
 int opt_tree_last_device_status(opt_tree_ctx* ctx, int32_t* status_host) {

@@ -54,7 +54,7 @@ __device__ __forceinline__ void pipeline_init(CtaSmem& s) {
 // Once a Source has said "no more work" no ticket of this CTA can still turn into a row.
 constexpr int kFetchLanes = 4;
 template <class Source>
-__device__ void fetcher_role(CtaSmem& s, Source& src, int* status) {
+__device__ void fetcher_role(CtaSmem& s, Source& src, int* status, long long limit = kWaitCycles) {
     const int lane = threadIdx.x & 31;
     const unsigned below = (1u << lane) - 1u;
     bool holding = false;                 // this lane has a ticket
@@ -100,7 +100,7 @@ __device__ void fetcher_role(CtaSmem& s, Source& src, int* status) {
         }
         if (rm) t0 = clock64();
         else {
-            if ((turn & 63) == 63 && clock64() - t0 > kWaitCycles) { set_status(status, kErrTimeout); return; }
+            if ((turn & 63) == 63 && clock64() - t0 > limit) { set_status(status, kErrTimeout); return; }
             __nanosleep(100);
         }
     }

@@ -147,15 +147,15 @@ __device__ __forceinline__ void stage_layer_candidates(LayerScratch& s, const Se
 
 // A candidate word that was not there yet when it was looked at is read again until it is (bounded).
 // Rare, so out of line.
-__device__ __noinline__ unsigned long long poll_phat_word(const unsigned long long* p, int* status) {
+__device__ __noinline__ unsigned long long poll_phat_word(const unsigned long long* p, int* status, int polls = kWaitPolls) {
     unsigned long long x = ld_relaxed_u64(p);
-    for (int t = 0; !(x >> 63) && t < (1 << 22); ++t) x = ld_relaxed_u64(p);
+    for (int t = 0; !(x >> 63) && t < polls; ++t) x = ld_relaxed_u64(p);
     if (!(x >> 63)) { set_status(status, kErrTimeout); x = ~0ull; }
     return x;
 }
-__device__ __noinline__ unsigned int poll_tok_word(const unsigned int* p, int* status) {
+__device__ __noinline__ unsigned int poll_tok_word(const unsigned int* p, int* status, int polls = kWaitPolls) {
     unsigned int x = ld_relaxed_u32(p);
-    for (int t = 0; !(x >> 31) && t < (1 << 22); ++t) x = ld_relaxed_u32(p);
+    for (int t = 0; !(x >> 31) && t < polls; ++t) x = ld_relaxed_u32(p);
     if (!(x >> 31)) { set_status(status, kErrTimeout); x = ~0u; }
     return x;
 }
