@@ -591,6 +591,49 @@ def parity_counts(g, o):
     return out
 
 
+def run_study(args):
+    """--study mal: acceptance length and E(A) of the adaptive tree against fixed trees of the same size on the
+    synthetic tables (paper_2406_17276_b200/study.py), one JSON line; the oracle on the first two steps' roots
+    beside it."""
+    import torch
+    from paper_2406_17276_b200 import build, study
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    build.build()
+    line = {"study": "mal", "data": "synthetic", "steps": args.steps,
+            "note": "acceptance length A counts the bonus token; E(A) of Eq. 3 does not, so E(A) + 1 is the figure to set against A",
+            "workloads": {}}
+    for nm in args.study_workloads.split(","):
+        res, first = study.run(nm, args.steps, keep_first=2)
+        if not args.no_cpu_baseline:
+            res["cpu_baseline"] = study_cpu_baseline(first)
+        line["workloads"][nm] = res
+    if args.budgets:
+        line["budget_sweep_c2"] = {str(n): study.run("c2", max(50, args.steps // 10), n=n)[0]["shapes"]
+                                   for n in (16, 64, 256, 512, 1000)}
+    print(json.dumps(line), flush=True)
+
+
+def study_cpu_baseline(first):
+    """The oracle on the first two steps' roots of a study: its acceptance lengths and E(A) beside the
+    library's for the same roots (both follow the same rule, so they agree up to near-ties)."""
+    import oracle
+    w, n = first["w"], first["n"]
+    ld, lt = first["tables"]
+    t0 = time.perf_counter()
+    oa, oe = [], []
+    for r in first["roots"]:
+        o = oracle.table_step(ld, lt, r, n, w.k, w.max_depth, NEG_INF)
+        oa.append(o.accept_len); oe.append(o.expected_len)
+    dt = time.perf_counter() - t0
+    oa, oe = np.array(oa), np.array(oe)
+    return {"kind": "oracle", "cores": 1, "sample": f"{len(first['roots'])} steps of {oa.shape[1]} sequences", "seconds": dt,
+            "value": oa.size / dt, "unit": UNIT,
+            "mean_acceptance_length": float(oa.mean()), "library_mean_acceptance_length_same_steps": float(first["A"].mean()),
+            "mean_expected_length": float(oe.mean()), "library_mean_expected_length_same_steps": float(first["E"].mean()),
+            "sequences_with_equal_acceptance_length": int((oa == first["A"]).sum()), "sequences": int(oa.size)}
+
+
 def run_reference(args):
     """The reference arm: the CPU oracle on the same config and metric (rank 0 only)."""
     if int(os.environ.get("RANK", 0)) != 0:
@@ -635,14 +678,15 @@ def main():
                     help="time the row step alone over this many rows instead of whole steps (its own roofline line)")
     ap.add_argument("--study", default=None, choices=["mal"],
                     help="mal: mean acceptance length and E(A) of OPT-Tree against fixed trees of the same size on the synthetic tables")
+    ap.add_argument("--study-workloads", default="c2,c4", help="workloads of --study, comma separated")
+    ap.add_argument("--budgets", action="store_true", help="--study: also sweep the node budget on c2 (16 ... 1000 nodes)")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.gpus > 1 and not shard.launched_by_torchrun():
             raise SystemExit(shard.launch_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
         run_reference(args)
     elif args.study:
-        from paper_2406_17276_b200 import study
-        study.main(args)
+        run_study(args)
     elif args.rows > 0:
         run_rows(args)
     else:

@@ -36,13 +36,13 @@ extern "C" {
 typedef enum {
     OPT_TREE_OK = 0,
     OPT_TREE_ERR_INVALID_ARG = -1,   /* null pointer, non-positive size, B > max_batch ... */
-    OPT_TREE_ERR_UNSUPPORTED = -2,   /* n > 256, k > 32, k > V, misaligned table ... */
+    OPT_TREE_ERR_UNSUPPORTED = -2,   /* n > 1024, k > 32, k > V, more than 510 layers ... */
     OPT_TREE_ERR_CUDA = -3,          /* a CUDA runtime call failed */
     OPT_TREE_ERR_TIMEOUT = -4,       /* a bounded device-side wait expired */
     OPT_TREE_ERR_INTERNAL = -5       /* a device-side bounds check failed */
 } opt_tree_status;
 
-#define OPT_TREE_MAX_N 256
+#define OPT_TREE_MAX_N 1024
 #define OPT_TREE_MAX_K 32
 
 typedef struct opt_tree_ctx opt_tree_ctx;   /* opaque; owns only its workspace */
@@ -52,7 +52,8 @@ typedef struct opt_tree_ctx opt_tree_ctx;   /* opaque; owns only its workspace *
  *   H          rows of the tables, H >= 1
  *   n          node budget of the tree (Algorithm 1 input n), 1 <= n <= OPT_TREE_MAX_N
  *   k          at most k children per node (the k most probable next tokens), 1 <= k <= OPT_TREE_MAX_K
- *   max_depth  cap on the number of drafted layers; Algorithm 1 also caps the depth by n
+ *   max_depth  cap on the number of drafted layers; Algorithm 1 also caps the depth by n;
+ *              min(max_depth, n) <= 510
  *   max_batch  largest B any call will pass */
 typedef struct {
     int32_t V, H, n, k, max_depth, max_batch;

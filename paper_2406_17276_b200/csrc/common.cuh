@@ -28,7 +28,7 @@ constexpr int kWarps = kConsumerWarps + kHelperWarps;
 constexpr int kThreads = kWarps * 32;               // 896 threads per CTA
 enum { kHelperIssuer = 0, kHelperFetcher = 1, kHelperLayer = 2, kHelperFirstAssistant = 3, kHelperFirstFinisher = 2 + kTeamWarps };
 constexpr int kMaxK = 32;
-constexpr int kMaxN = 256;
+constexpr int kMaxN = 1024;
 
 // Device status codes mirror opt_tree_status.
 constexpr int kErrTimeout = -4;

@@ -161,11 +161,12 @@ __device__ __forceinline__ TreeOut tree_out(const opt_tree_out& o, const Params&
     return t;
 }
 
-// Mailbox item: bit 63 valid | b (15 bits) | layer d (9) | frontier slot (8) | table row of the node to
+// Mailbox item: bit 63 valid | b (15 bits) | layer d (9) | void flag (1) | frontier slot (10, from bit 22) | table row of the node to
 // expand (22).  A second word at the same mailbox position carries the node's path value (bit 63
 // valid; a path value is never negative).  Both words validate themselves, so a row can be expanded
 // from them alone and the publisher needs no fence before writing them.
 constexpr int kMaxTableRows = 1 << 22;
+constexpr int kMaxLayers = 510;             // layers a build may draft: layer d+1 must fit the item's 9-bit field
 __device__ __forceinline__ unsigned long long item_encode(int b, int d, int slot, int row) {
     return (1ull << 63) | ((unsigned long long)b << 48) | ((unsigned long long)d << 39) |
            ((unsigned long long)slot << 22) | (unsigned long long)row;
@@ -227,7 +228,7 @@ struct BuildSource {
         if (!((item & ph) >> 63)) return check_done && ld_acquire_s32(&w.q_ctl[kQDone]) ? -1 : 0;
         if (kPrune && (item & kItemVoid)) return 2;
         d.b = (int)((item >> 48) & 0x7FFFu); d.d = (int)((item >> 39) & 0x1FFu);
-        d.slot = (int)((item >> 22) & 0xFFu); d.fsize = 0;
+        d.slot = (int)((item >> 22) & 0x3FFu); d.fsize = 0;
         d.pphat = __longlong_as_double((long long)(ph & 0x7FFFFFFFFFFFFFFFull));
         int row = (int)(item & 0x3FFFFFu);
         if (row >= p.H) { set_status(w.status, kErrInternal); row = 0; }
@@ -387,7 +388,7 @@ struct BuildSink {
             const LayerJob j = ls.job;
             if (j.kind == 0) return;
             if (j.kind == 2) select_running_team(ls, j, tt, w.status);
-            else if (j.fsize * j.k <= 1024) select_layer_team<kPrune>(ls, j, tt, w.status);
+            else if (j.fsize * j.k <= kStageCap) select_layer_team<kPrune>(ls, j, tt, w.status);
             else select_layer_team_big<kPrune>(ls, j, tt, w.status);
         }
     }
@@ -426,7 +427,7 @@ struct BuildSink {
                     if (kPrune || d == p.Dcap) {
                         const int nR_old = d == 1 ? 0 : __ldcg(&sw.st[kStNR]);
                         const int off = (nR_old + 1) & ~1;
-                        if (off + fsize * p.k <= 1024) {
+                        if (off + fsize * p.k <= kStageCap) {
                             const int sent = merged_layer_job(ls, sw, b, d, fsize, nR_old, off);
                             if (sent > 0) { cur_d[q] = d + 1; cur_f[q] = sent; cur_tot[q] += sent; }
                             if (kPrune && lane == 0) sw.st[kStRows] = cur_tot[q];
@@ -444,7 +445,7 @@ struct BuildSink {
                     unsigned g0 = 0;
                     if (early) g0 = reserve_layer(nl);        // the rows' numbers, while the candidates load
                     {
-                        const bool small = fsize * p.k <= 1024;    // the candidates fit the shared-memory staging
+                        const bool small = fsize * p.k <= kStageCap;    // the candidates fit the shared-memory staging
                         if (lane == 0) {
                             LayerJob& j = ls.job;
                             j.kind = 1; j.d = d; j.fsize = fsize; j.n = p.n; j.k = p.k; j.kk = p.kk;
@@ -519,7 +520,7 @@ build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, opt_tree
     CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
     BuildSource<kPrune> src{w, p, draft};
     BuildSink<kPrune> sink{w, p, out};
-    run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, w.status);
+    run_pipeline(s, src, sink, p.V, p.k, p.n, p.aligned != 0, w.status);
 }
 
 // The row step alone over a list of rows (static round-robin over the CTAs).
@@ -556,7 +557,7 @@ row_topk_kernel(Params p, const uint16_t* __restrict__ logits, const int32_t* __
     CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
     ListSource src{logits, rows, nrows, p.V, p.H, (int)blockIdx.x, (int)gridDim.x, status};
     ListSink sink{tok_out, prob_out, p.k};
-    run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, status);
+    run_pipeline(s, src, sink, p.V, p.k, p.n, p.aligned != 0, status);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -581,6 +582,8 @@ __global__ void __launch_bounds__(kTeam)
 layer_step_kernel(Workspace w, Params p, int fstride, opt_tree_out out, int32_t* next_tokens, int32_t* next_parent,
                   int32_t* next_count) {
     __shared__ LayerScratch ls;
+    extern __shared__ __align__(16) unsigned char ls_tail[];       // the n-sized arrays (layer_tail_bytes(n))
+    if (threadIdx.x == 0) layer_tail_carve(ls, ls_tail, p.n);
     grid_dependency_wait();
     const int b = blockIdx.x, tt = threadIdx.x, lane = tt & 31;
     for (int i = tt; i < 3 * 256; i += kTeam) (&ls.thist[0][0])[i] = 0;
@@ -603,7 +606,7 @@ layer_step_kernel(Workspace w, Params p, int fstride, opt_tree_out out, int32_t*
         reinterpret_cast<unsigned int*>(sw.cand_tok)[i] = valid ? (0x80000000u | (unsigned int)tok) : ~0u;
     }
     __syncthreads();
-    const bool small = N <= 1024;
+    const bool small = N <= kStageCap;
     if (tt < 32 && small) { stage_layer_candidates(ls, sw, fsize, p.k); cp_async_wait_all(); }
     if (tt == 0) {
         LayerJob& j = ls.job;
@@ -630,34 +633,38 @@ layer_step_kernel(Workspace w, Params p, int fstride, opt_tree_out out, int32_t*
     }
 }
 
-// Tree attention mask + position ids: one CTA per sequence, one thread per node.
+// Tree attention mask + position ids: one CTA per sequence, a thread per node (in rounds of the block
+// size when n is larger): the node's ancestor chain is walked and its bits gathered in registers.
 __global__ void __launch_bounds__(kSmallThreads)
 mask_kernel(const int32_t* __restrict__ parent, const int32_t* __restrict__ depth, const int32_t* __restrict__ n_sel,
             const int32_t* __restrict__ base_pos, int n, uint64_t* mask, int32_t* position_ids, int* status) {
     grid_dependency_wait();
-    const int b = blockIdx.x, i = threadIdx.x;
-    if (i >= n) return;
+    const int b = blockIdx.x;
     const int W = (n + 63) >> 6;
     const int ns = n_sel[b];
     const int32_t* par = parent + (size_t)b * n;
-    uint64_t bits[kMaxN / 64] = {0, 0, 0, 0};
-    int pos = 0;
-    if (i < ns) {
-        int a = i, steps = 0;
-        while (a >= 0 && steps <= n) {                      // an ancestor chain is at most n long
-            if (a >= n) { set_status(status, kErrInternal); break; }
+    for (int i = threadIdx.x; i < n; i += kSmallThreads) {
+        uint64_t bits[kMaxN / 64];
 #pragma unroll
-            for (int wd = 0; wd < kMaxN / 64; ++wd)
-                if ((a >> 6) == wd) bits[wd] |= 1ull << (a & 63);
-            a = par[a];
-            ++steps;
+        for (int wd = 0; wd < kMaxN / 64; ++wd) bits[wd] = 0ull;
+        int pos = 0;
+        if (i < ns) {
+            int a = i, steps = 0;
+            while (a >= 0 && steps <= n) {                  // an ancestor chain is at most n long
+                if (a >= n) { set_status(status, kErrInternal); break; }
+#pragma unroll
+                for (int wd = 0; wd < kMaxN / 64; ++wd)
+                    if ((a >> 6) == wd) bits[wd] |= 1ull << (a & 63);
+                a = par[a];
+                ++steps;
+            }
+            pos = (base_pos ? base_pos[b] : 0) + depth[(size_t)b * n + i];
         }
-        pos = (base_pos ? base_pos[b] : 0) + depth[(size_t)b * n + i];
-    }
 #pragma unroll
-    for (int wd = 0; wd < kMaxN / 64; ++wd)
-        if (wd < W) mask[((size_t)b * n + i) * W + wd] = bits[wd];
-    position_ids[(size_t)b * n + i] = pos;
+        for (int wd = 0; wd < kMaxN / 64; ++wd)
+            if (wd < W) mask[((size_t)b * n + i) * W + wd] = bits[wd];
+        position_ids[(size_t)b * n + i] = pos;
+    }
 }
 
 // After verification: the bitmask expanded to the dense (n+1) x (n+1) form, position 0 being the
@@ -960,7 +967,7 @@ __global__ void __launch_bounds__(kThreads)
 wait_probe_kernel(int* result, const unsigned long long* zero_words, long long limit, int polls) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
-    pipeline_init(s);
+    pipeline_init(s, 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp == 0) {
         mbar_wait_warp(&s.full_bar[0], 0u, &result[0], limit);
@@ -988,6 +995,7 @@ struct opt_tree_ctx {
     size_t bytes;
     int device;
     int grid;              // resident CTAs of the persistent kernels (SMs x occupancy)
+    size_t smem;           // dynamic shared memory of one such CTA (cta_smem_bytes(cfg.n))
     int mcap;
     int64_t launches;
     // pinned host staging of opt_tree_step_host: the step's inputs and outputs cross the bus in one
@@ -1005,6 +1013,7 @@ int supported_cfg(const opt_tree_config* c) {
     if (c->n > OPT_TREE_MAX_N || c->k > OPT_TREE_MAX_K || c->k > c->V) return OPT_TREE_ERR_UNSUPPORTED;
     if ((long long)c->V * 31 + c->max_depth > 2147483647LL) return OPT_TREE_ERR_UNSUPPORTED;
     if (c->max_batch > 32767 || c->max_depth > 65535 || c->H > ot::kMaxTableRows) return OPT_TREE_ERR_UNSUPPORTED;
+    if ((c->max_depth < c->n ? c->max_depth : c->n) > ot::kMaxLayers) return OPT_TREE_ERR_UNSUPPORTED;   // the mailbox item's layer field
     return OPT_TREE_OK;
 }
 ot::Params make_params(const opt_tree_ctx* ctx, const void* table, float delta) {
@@ -1045,13 +1054,19 @@ extern "C" {
 
 // CTAs of the persistent kernels on the current device (one CTA of kThreads per SM as long as its
 // shared memory fits); 0 if there is no usable device.
-static int persistent_grid() {
+// Shared memory of a CTA of the persistent kernels for node budget n: the fixed part and the layer team's
+// n-sized arrays behind it.
+static size_t cta_smem_bytes(int n) { return sizeof(ot::CtaSmem) + ((ot::layer_tail_bytes(n) + 15) & ~(size_t)15); }
+
+static int persistent_grid(int n) {
     int dev = 0, per_sm = 0, sms = 0;
+    const int most = (int)cta_smem_bytes(OPT_TREE_MAX_N);
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
-    if (cudaFuncSetAttribute(ot::build_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
-        cudaFuncSetAttribute(ot::build_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
-        cudaFuncSetAttribute(ot::row_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ot::build_kernel<true>, ot::kThreads, sizeof(ot::CtaSmem)) != cudaSuccess ||
+    if (cudaFuncSetAttribute(ot::build_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::build_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::row_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::layer_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ot::layer_tail_bytes(OPT_TREE_MAX_N)) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ot::build_kernel<true>, ot::kThreads, cta_smem_bytes(n)) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
         cudaGetLastError();
         return 0;
@@ -1062,7 +1077,7 @@ static int persistent_grid() {
 
 size_t opt_tree_workspace_bytes(const opt_tree_config* cfg) {
     if (!valid_cfg(cfg) || supported_cfg(cfg) != OPT_TREE_OK) return 0;
-    int grid = persistent_grid();
+    int grid = persistent_grid(cfg->n);
     if (grid == 0) grid = 148;                       // no device here: the size on a B200
     return ot::carve(*cfg, grid, nullptr, nullptr);
 }
@@ -1077,7 +1092,8 @@ int opt_tree_create(opt_tree_ctx** out, const opt_tree_config* cfg) {
     if (!ctx) return OPT_TREE_ERR_CUDA;
     ctx->cfg = *cfg;
     ctx->launches = 0;
-    ctx->grid = persistent_grid();
+    ctx->grid = persistent_grid(cfg->n);
+    ctx->smem = cta_smem_bytes(cfg->n);
     if (ctx->grid == 0) { delete ctx; return OPT_TREE_ERR_CUDA; }
     ctx->mcap = (int)ot::mailbox_capacity(*cfg, ctx->grid);
     ctx->bytes = ot::carve(*cfg, ctx->grid, nullptr, nullptr);
@@ -1122,10 +1138,10 @@ static int build_common(opt_tree_ctx* ctx, const void* draft, const int32_t* roo
     const long long init_threads = (long long)ctx->grid * ctx->mcap > B ? (long long)ctx->grid * ctx->mcap : B;
     launch_after(ot::init_build_kernel, dim3((unsigned)((init_threads + 255) / 256)), dim3(256), 0, st, ctx->ws, p, root_token);
     if (prune)
-        launch_after(ot::build_kernel<true>, dim3(ctx->grid), dim3(ot::kThreads), sizeof(ot::CtaSmem), st,
+        launch_after(ot::build_kernel<true>, dim3(ctx->grid), dim3(ot::kThreads), ctx->smem, st,
                      ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
     else
-        launch_after(ot::build_kernel<false>, dim3(ctx->grid), dim3(ot::kThreads), sizeof(ot::CtaSmem), st,
+        launch_after(ot::build_kernel<false>, dim3(ctx->grid), dim3(ot::kThreads), ctx->smem, st,
                      ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
     ctx->launches += 2;
     int rc = check_launch();
@@ -1215,10 +1231,10 @@ int opt_tree_layers_step(opt_tree_ctx* ctx, const void* frontier_logits, int32_t
     ot::Params pr = p;
     pr.H = nrows;                                            // the dense buffer is the "table" of the row step
     const int grid = nrows < ctx->grid ? nrows : ctx->grid;
-    launch_after(ot::row_topk_kernel, dim3(grid), dim3(ot::kThreads), sizeof(ot::CtaSmem), st,
+    launch_after(ot::row_topk_kernel, dim3(grid), dim3(ot::kThreads), ctx->smem, st,
                  pr, static_cast<const uint16_t*>(frontier_logits), static_cast<const int32_t*>(nullptr), nrows, ctx->ws.rtok,
                  ctx->ws.rprob, ctx->ws.status);
-    launch_after(ot::layer_step_kernel, dim3(B), dim3(ot::kTeam), 0, st, ctx->ws, p, frontier_stride, *out, next_tokens,
+    launch_after(ot::layer_step_kernel, dim3(B), dim3(ot::kTeam), ot::layer_tail_bytes(ctx->cfg.n), st, ctx->ws, p, frontier_stride, *out, next_tokens,
                  next_parent, next_count);
     ctx->launches += 2;
     return check_launch();
@@ -1230,7 +1246,7 @@ int opt_tree_row_softmax_topk(opt_tree_ctx* ctx, const void* logits, const int32
     if (nrows == 0) return OPT_TREE_OK;
     const ot::Params p = make_params(ctx, logits, 0.0f);
     const int grid = nrows < ctx->grid ? nrows : ctx->grid;
-    ot::row_topk_kernel<<<grid, ot::kThreads, sizeof(ot::CtaSmem), static_cast<cudaStream_t>(stream)>>>(
+    ot::row_topk_kernel<<<grid, ot::kThreads, ctx->smem, static_cast<cudaStream_t>(stream)>>>(
         p, static_cast<const uint16_t*>(logits), rows, nrows, tok_out, prob_out, ctx->ws.status);
     ctx->launches++;
     return check_launch();
@@ -1272,13 +1288,13 @@ int opt_tree_step_host(opt_tree_ctx* ctx, const void* draft, const void* target,
 int opt_tree_selftest_waits(opt_tree_ctx* ctx, int32_t* result, void* stream) {
     if (!ctx || !result) return OPT_TREE_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaFuncSetAttribute(ot::wait_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
+    if (cudaFuncSetAttribute(ot::wait_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cta_smem_bytes(1)) != cudaSuccess ||
         cudaMemsetAsync(result, 0, OPT_TREE_SELFTEST_WAITS * sizeof(int32_t), st) != cudaSuccess ||
         cudaMemsetAsync(ctx->ws.rprob, 0, 2 * sizeof(unsigned long long), st) != cudaSuccess) {     // two words nobody writes
         cudaGetLastError();
         return OPT_TREE_ERR_CUDA;
     }
-    ot::wait_probe_kernel<<<1, ot::kThreads, sizeof(ot::CtaSmem), st>>>(
+    ot::wait_probe_kernel<<<1, ot::kThreads, cta_smem_bytes(1), st>>>(
         result, reinterpret_cast<const unsigned long long*>(ctx->ws.rprob), 1ll << 16, 1 << 10);
     ctx->launches++;
     return check_launch();

@@ -28,8 +28,10 @@
 
 namespace ot {
 
-__device__ __forceinline__ void pipeline_init(CtaSmem& s) {
+// n: the context's node budget; the layer team's n-sized arrays start right behind the CtaSmem.
+__device__ __forceinline__ void pipeline_init(CtaSmem& s, int n) {
     if (threadIdx.x == 0) {
+        layer_tail_carve(s.layer, reinterpret_cast<unsigned char*>(&s) + sizeof(CtaSmem), n);
         for (int i = 0; i < kStages; ++i) { mbar_init(&s.full_bar[i], 1); mbar_init(&s.empty_bar[i], kConsumerWarps); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(&s.ready_bar[i], kConsumerWarps); mbar_init(&s.free_bar[i], 1); }
         for (int i = 0; i < kDesc; ++i) { mbar_init(&s.desc_full[i], 1); mbar_init(&s.desc_empty[i], kConsumerWarps); }
@@ -222,8 +224,8 @@ __device__ void finisher_role(CtaSmem& s, Sink& sink, int fidx, int V, int k, bo
 }
 
 template <class Source, class Sink>
-__device__ __forceinline__ void run_pipeline(CtaSmem& s, Source& src, Sink& sink, int V, int k, bool aligned, int* status) {
-    pipeline_init(s);
+__device__ __forceinline__ void run_pipeline(CtaSmem& s, Source& src, Sink& sink, int V, int k, int n, bool aligned, int* status) {
+    pipeline_init(s, n);
     grid_dependency_wait();                                // shared memory is set up; global memory from here on
     const int warp = threadIdx.x >> 5;
     if (warp < kConsumerWarps) { consumer_role(s, warp, V, status); return; }

@@ -80,14 +80,19 @@ struct LayerJob {                  // what the layer warp hands its assistants (
     int32_t* Rnew;                 // the new top-n's gids, ascending
 };
 
-struct alignas(16) LayerScratch {  // private to the layer team of a CTA
-    unsigned long long keys[1024 + 2];         // staged candidate keys, then the keys of R + layer
-    unsigned long long lkeys[kMaxN];           // keys of the new layer, slot order
-    double vals[kMaxN];                        // path values of the new running top-n
-    int toks[1024 + 4];                        // staged candidate tokens
-    int gids[2 * kMaxN];
-    int rsel[kMaxN];                           // gids of the new running top-n, ascending
-    int ltok[kMaxN];                           // tokens of the new layer, slot order
+constexpr int kStageCap = 1024;                    // candidates of a layer that the shared-memory staging holds
+
+// Private to the layer team of a CTA.  The arrays whose length follows the node budget n are not
+// members: they live behind the CTA's fixed shared memory, sized by the context's n (see
+// layer_tail_bytes / layer_tail_carve), so that a small n keeps the CTA's shared memory small.
+struct alignas(16) LayerScratch {
+    unsigned long long* keys;                  // [max(kStageCap, 2n) + 2] staged candidate keys, then the keys of R + layer
+    unsigned long long* lkeys;                 // [n]  keys of the new layer, slot order
+    double* vals;                              // [n]  path values of the new running top-n
+    int* gids;                                 // [2n]
+    int* rsel;                                 // [n]  gids of the new running top-n, ascending
+    int* ltok;                                 // [n]  tokens of the new layer, slot order
+    int toks[kStageCap + 4];                   // staged candidate tokens
     int hist[256];
     int thist[3][256];                         // the team's digit counts, rotating (all zero between selections)
     unsigned long long red_or[kTeamWarps], red_and[kTeamWarps];
@@ -118,6 +123,21 @@ struct alignas(128) CtaSmem {
     unsigned long long desc_empty[kDesc];      // consumers -> fetcher (descriptor may be overwritten)
     volatile int stop_row;                     // first row index that is the stop marker
 };
+
+// Bytes of the n-sized arrays of LayerScratch, and their placement behind `base` (16-byte aligned).
+__host__ __device__ inline size_t layer_tail_bytes(int n) {
+    const size_t nk = (size_t)(2 * n > kStageCap ? 2 * n : kStageCap) + 2;
+    return nk * 8 + (size_t)n * 8 * 2 + (size_t)n * 4 * 4;
+}
+__device__ __forceinline__ void layer_tail_carve(LayerScratch& s, unsigned char* base, int n) {
+    const size_t nk = (size_t)(2 * n > kStageCap ? 2 * n : kStageCap) + 2;
+    s.keys = reinterpret_cast<unsigned long long*>(base);
+    s.lkeys = s.keys + nk;
+    s.vals = reinterpret_cast<double*>(s.lkeys + n);
+    s.gids = reinterpret_cast<int*>(s.vals + n);
+    s.rsel = s.gids + 2 * n;
+    s.ltok = s.rsel + n;
+}
 
 __device__ __forceinline__ int chunk_elems(int V, int c) {
     int rem = V - c * kChunkElems;

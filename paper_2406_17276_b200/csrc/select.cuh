@@ -136,7 +136,7 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
 __device__ __forceinline__ void stage_layer_candidates(LayerScratch& s, const SeqWork& w, int fsize, int k, int off = 0) {
     const int lane = threadIdx.x & 31;
     const int N = fsize * k;
-    if (off + N > 1024) return;                            // (off is even: the copies keep their 16-byte alignment)
+    if (off + N > kStageCap) return;                       // (off is even: the copies keep their 16-byte alignment)
     const unsigned long long* gph = reinterpret_cast<const unsigned long long*>(w.cand_phat);
     const unsigned int* gtk = reinterpret_cast<const unsigned int*>(w.cand_tok);
     #pragma unroll 1
@@ -589,7 +589,7 @@ __device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork&
     // --- E_sub(T, n): the n largest path values among the previous top-n and the new layer ---
     const int32_t* Rold = w.R + ((d - 1) & 1) * n;
     int32_t* Rnew = w.R + (d & 1) * n;
-    const int NR = nR_old + nl;                           // <= 2n <= 512
+    const int NR = nR_old + nl;                           // <= 2n
     const int nR = NR < n ? NR : n;
     unsigned long long ko = 0ull, ka = ~0ull;
     #pragma unroll 1

@@ -33,6 +33,8 @@ def test_host_only_entry_points_work_without_a_gpu():
     assert L.opt_tree_strerror(-4) == b"device-side wait timed out"
     good = binding.Config(32000, 4096, 64, 10, 10, 32)
     assert L.opt_tree_workspace_bytes(good) > 0
-    assert L.opt_tree_workspace_bytes(binding.Config(32000, 4096, 257, 10, 10, 32)) == 0
+    assert L.opt_tree_workspace_bytes(binding.Config(32000, 4096, 1024, 32, 20, 8)) > 0
+    assert L.opt_tree_workspace_bytes(binding.Config(32000, 4096, 1025, 10, 10, 32)) == 0
+    assert L.opt_tree_workspace_bytes(binding.Config(32000, 4096, 1024, 10, 511, 32)) == 0      # more layers than a mailbox item can name
     assert L.opt_tree_workspace_bytes(binding.Config(32000, 4096, 64, 33, 10, 32)) == 0
     assert L.opt_tree_workspace_bytes(None) == 0

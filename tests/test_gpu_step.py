@@ -62,6 +62,16 @@ def test_degenerate_and_maximum_sizes(request, n, k, D, B, V):
     assert t["exact"] > 0 and t["near_tie"] + t["stop_near_tie"] <= 0.05 * (t["exact"] + 1)
 
 
+@pytest.mark.parametrize("n,k,D,B", [(512, 16, 10, 4), (512, 32, 8, 3), (1000, 16, 8, 3), (1000, 32, 6, 2), (1024, 32, 12, 2), (300, 4, 24, 1)])
+def test_node_budgets_beyond_256(request, n, k, D, B):
+    """Trees of several hundred to a thousand nodes (the paper's Section 4.3 grows its trees past 500 nodes):
+    V = 32000, a table of 512 rows so that the oracle's row memo keeps the comparison short."""
+    w = synth.Workload("large_n", B, 32000, n, k, D, 3.0, 1.1, 0.2, H=512, seed=n + k)
+    t = _run(w, [NEG_INF, 0.05], steps=2)
+    record_parity(request.node.nodeid, t)
+    assert t["exact"] > 0 and t["near_tie"] + t["stop_near_tie"] <= 0.05 * (t["exact"] + 1)
+
+
 def test_two_runs_are_bit_identical():
     w = synth.WORKLOADS["c4"]
     ld, lt = synth.make_tables(w, H=256, V=20000)
@@ -99,7 +109,7 @@ def test_host_buffer_step_matches_device_path():
 
 def test_argument_checks_return_status_codes():
     with pytest.raises(binding.OptTreeError) as e:
-        binding.OptTree(32000, 64, 257, 10, 10, 1)
+        binding.OptTree(32000, 64, 1025, 10, 10, 1)
     assert e.value.code == binding.ERR_UNSUPPORTED
     with pytest.raises(binding.OptTreeError) as e:
         binding.OptTree(32000, 64, 64, 33, 10, 1)

@@ -9,7 +9,7 @@ from tests import _defs
 NEG_INF = float("-inf")
 
 
-@pytest.mark.parametrize("n,k,D", [(10, 10, 6), (64, 10, 10), (100, 8, 12), (256, 32, 20)])
+@pytest.mark.parametrize("n,k,D", [(10, 10, 6), (64, 10, 10), (100, 8, 12), (256, 32, 20), (512, 16, 10), (1000, 32, 8)])
 def test_mask_is_ancestor_or_self_by_parent_walk(n, k, D):
     tab = _defs.small_table(128, 1024, 31)
     base = np.array([7, 1000], np.int32)
