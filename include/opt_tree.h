@@ -196,8 +196,11 @@ int opt_tree_layers_step(opt_tree_ctx *ctx, const void *frontier_logits_bf16, in
  * Randomness is reproducible: one uniform per (sequence b, position j; 0 = root, i+1 = node i) from the
  * counter-based generator Philox4x32-10 (Salmon et al., 2011) with key = seed and counter =
  * (j, b, step low word, step high word), u = top 53 bits of the first two output words * 2^-53; the
- * draw is by inverse CDF in token order on e_v = exp((x_v - max x) / tau) in double precision (the
- * first token whose running sum exceeds u * sum; the last token with e_v > 0 if rounding leaves none).
+ * draw is by inverse CDF in token order on e_v = exp((x_v - max x) / tau): the first token whose running
+ * sum exceeds u * sum (the last token with e_v > 0 if rounding leaves none).  The row is read once: the
+ * running sum is formed per segment of 512 logits in single precision (exponent arithmetic exact for
+ * bf16 logits), and in double precision inside the segment where u * sum falls, so the token is that of
+ * a double-precision inverse CDF unless u * sum lies within about 1e-6 * sum of a running sum.
  * `step` is the caller's decoding step number, so that successive steps use fresh uniforms.
  * Errors as opt_tree_verify; tau <= 0 or NaN is OPT_TREE_ERR_INVALID_ARG. */
 int opt_tree_verify_sampled(opt_tree_ctx *ctx, const opt_tree_out *tree, const void *target_logits_bf16,

@@ -849,14 +849,98 @@ __device__ __forceinline__ double uniform53(unsigned long long seed, unsigned lo
     return (double)bits * (1.0 / 9007199254740992.0);
 }
 
+// Sampling works on segments of 64 vectors (512 logits): one warp, two coalesced 16-byte loads per lane.
+constexpr int kSegVecs = 64;
+constexpr int kSegTokens = kSegVecs * 8;
+constexpr int kMaxSeg = 640;                 // rows of up to 327 680 logits take the one-pass path
+constexpr int kSampleExpLimit = 1 << 22;     // |exponent| beyond which the single-precision pass cannot scale
+struct alignas(8) SegPart { float sum; int E; };       // a segment's sum of 2^(x*c - E), E an integer
 struct SampleSmem {
+    union { SegPart part[kMaxSeg]; double cum[kMaxSeg]; };   // per segment: its partial sum, then the running sum up to and including it
     double wsum[kVerifyThreads / 32];
+    double S;
     float wmax[kVerifyThreads / 32];
-    int chosen, last_live;
+    int wE[kVerifyThreads / 32];
+    int chosen, last_live, seg, live_seg;
 };
 
-// CTA (j, b) as in verify_kernel.  Thread t owns the tokens [t*L, (t+1)*L): its own sum, a scan over the
-// threads in token order, and the thread in whose stretch u*S falls walks it once more.
+// The plain way, for rows the one-pass path does not take (unaligned rows, very long rows, extreme
+// magnitudes): thread t owns the tokens [t*L, (t+1)*L); the row's maximum, then every thread's sum of
+// double-precision exponentials in token order, a scan over the threads, and the thread in whose stretch
+// u*S falls walks it once more.  Returns the drawn token to every thread.
+__device__ __noinline__ int sample_row_plain(SampleSmem& q, const uint16_t* row, int V, bool vec, double tau, double u) {
+    const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
+    const int L = (((V + kVerifyThreads - 1) / kVerifyThreads) + 7) & ~7;       // tokens per thread, a multiple of 8
+    const int lo = min(tid * L, V), hi = min(lo + L, V);
+    auto logit = [&](int v) -> float { return bf16_bits_to_float(__ldg(row + v)); };
+    const uint4* rv = reinterpret_cast<const uint4*>(row);
+    float mx = -INFINITY;
+    if (vec) {
+        for (int v8 = lo >> 3; v8 < hi >> 3; ++v8) {
+            const uint4 x = ld_nc_v4(rv + v8);
+            const uint32_t m2 = max_bf16x2(max_bf16x2(x.x, x.y), max_bf16x2(x.z, x.w));
+            mx = fmaxf(mx, fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u)));
+        }
+    } else {
+        for (int v = lo; v < hi; ++v) mx = fmaxf(mx, logit(v));
+    }
+    mx = warp_max_f32(mx);
+    __syncthreads();                                         // (the scratch may still be in use by the one-pass path)
+    if (lane == 0) q.wmax[wp] = mx;
+    if (tid == 0) { q.chosen = -1; q.last_live = -1; }
+    __syncthreads();
+    mx = q.wmax[0];
+#pragma unroll
+    for (int i = 1; i < kVerifyThreads / 32; ++i) mx = fmaxf(mx, q.wmax[i]);
+    const double m = (double)mx;
+    double mine = 0.0;
+    int live = -1;                                           // last token of the stretch with a positive term
+    for (int v = lo; v < hi; ++v) {
+        const double e = exp(((double)logit(v) - m) / tau);
+        mine += e;
+        if (e > 0.0) live = v;
+    }
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) q.wsum[wp] = incl;
+    __syncthreads();
+    double base = 0.0, S = 0.0;                              // running sums before this warp / of the row, added up in one fixed order
+#pragma unroll
+    for (int i = 0; i < kVerifyThreads / 32; ++i) { if (i == wp) base = S; S += q.wsum[i]; }
+    // a thread's stretch begins exactly where the previous thread's ends: the same expression on both sides
+    double prev = __shfl_up_sync(0xFFFFFFFFu, incl, 1);
+    if (lane == 0) prev = 0.0;
+    const double excl_t = base + prev, incl_t = base + incl;
+    const double t = u * S;
+    atomicMax(&q.last_live, live);
+    if (incl_t > t && !(excl_t > t) && hi > lo) {            // the stretch in which the running sum passes t: one thread
+        double run = excl_t;
+        int y = live;
+        for (int v = lo; v < hi; ++v) {
+            run += exp(((double)logit(v) - m) / tau);
+            if (run > t) { y = v; break; }
+        }
+        atomicMax(&q.chosen, y);
+    }
+    __syncthreads();
+    int y = q.chosen;
+    if (y < 0) y = q.last_live < 0 ? 0 : q.last_live;        // rounding left no stretch: the last token with a positive term
+    return y;
+}
+
+// CTA (j, b) as in verify_kernel.  One pass over the row: warp w takes the segments w, w + 4, ...; a
+// segment's terms 2^(x*c - E) (c = log2(e) / tau, E an integer just above the segment's largest exponent)
+// are summed in single precision with ex2.approx and kept per segment, so the running sum is known in
+// token order at segment granularity.  The exponent x*c is formed with c split into a 16-bit head and a
+// tail: x is bf16, so x * head is exact, and the rounding of c does not grow with |x*c| (low temperatures).
+// Then: a double-precision scan over the segments, the segment in which u*S falls, and inside that segment
+// (512 logits, four per thread) double-precision exponentials and an exact scan.  What can differ from a
+// double-precision inverse CDF over the whole row is the placement of u*S relative to a segment's start, by
+// the rounding of the single-precision sums (a few 1e-7 of S).
 __global__ void __launch_bounds__(kVerifyThreads)
 verify_sampled_kernel(Workspace w, Params p, const uint16_t* __restrict__ target, const int32_t* __restrict__ root_token,
                       opt_tree_out tree, double tau, unsigned long long seed, unsigned long long step, int32_t* accept_len,
@@ -873,82 +957,132 @@ verify_sampled_kernel(Workspace w, Params p, const uint16_t* __restrict__ target
     const int depth = j == 0 ? 0 : tree.depth[(size_t)b * p.n + j - 1];
     if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
     const uint16_t* row = target + (size_t)row_of(token, depth, p.H) * p.V;
-    const int L = (((p.V + kVerifyThreads - 1) / kVerifyThreads) + 7) & ~7;       // tokens per thread, a multiple of 8
-    const int lo = min(tid * L, p.V), hi = min(lo + L, p.V);
-    auto logit = [&](int v) -> float { return bf16_bits_to_float(__ldg(row + v)); };
-    const bool vec = p.aligned != 0;                         // then a stretch starts on a 16-byte boundary and V is a multiple of 8
-    const uint4* rv = reinterpret_cast<const uint4*>(row);
-
-    // the row's maximum
-    float mx = -INFINITY;
-    if (vec) {
-        for (int v8 = lo >> 3; v8 < hi >> 3; ++v8) {
-            const uint4 x = ld_nc_v4(rv + v8);
-            const uint32_t m2 = max_bf16x2(max_bf16x2(x.x, x.y), max_bf16x2(x.z, x.w));
-            mx = fmaxf(mx, fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u)));
-        }
-    } else {
-        for (int v = lo; v < hi; ++v) mx = fmaxf(mx, logit(v));
-    }
-    mx = warp_max_f32(mx);
-    if (lane == 0) q.wmax[wp] = mx;
-    if (tid == 0) { q.chosen = -1; q.last_live = -1; }
-    __syncthreads();
-    mx = q.wmax[0];
+    const double u = uniform53(seed, step, b, j);
+    const int nv = p.V >> 3, nseg = (nv + kSegVecs - 1) / kSegVecs;
+    const double c64 = kLog2eD / tau;
+    bool fast = p.aligned != 0 && nseg <= kMaxSeg && c64 < 1e30;
+    int y = 0;
+    if (fast) {
+        const float c32 = (float)c64;
+        const float c_hi = __uint_as_float(__float_as_uint(c32) & 0xFFFFFF00u);      // 16 significant bits
+        const float c_lo = (float)(c64 - (double)c_hi);
+        const uint4* rv = reinterpret_cast<const uint4*>(row);
+        if (tid == 0) { q.chosen = -1; q.last_live = -1; q.seg = 0x7FFFFFFF; q.live_seg = -1; }
+#pragma unroll 1
+        for (int sg = wp; sg < nseg; sg += kVerifyThreads / 32) {
+            const int v0 = sg * kSegVecs + lane, v1 = v0 + 32;
+            const uint4 pad = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+            const uint4 q0 = v0 < nv ? ld_nc_v4(rv + v0) : pad, q1 = v1 < nv ? ld_nc_v4(rv + v1) : pad;
+            uint32_t ww[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+            uint32_t m2 = ww[0];
 #pragma unroll
-    for (int i = 1; i < kVerifyThreads / 32; ++i) mx = fmaxf(mx, q.wmax[i]);
-    const double m = (double)mx, inv_tau = 1.0 / tau;
-
-    // this thread's sum in token order, then the sums before it
-    double mine = 0.0;
-    int live = -1;                                           // last token of the stretch with a positive term
-    if (vec) {
-        for (int v8 = lo >> 3; v8 < hi >> 3; ++v8) {
-            const uint4 x = ld_nc_v4(rv + v8);
-            const uint32_t ww[4] = {x.x, x.y, x.z, x.w};
+            for (int i = 1; i < 8; ++i) m2 = max_bf16x2(m2, ww[i]);
+            const uint32_t wkey = __reduce_max_sync(0xFFFFFFFFu, max(ord16(m2 & 0xFFFFu), ord16(m2 >> 16)));
+            float sum = 0.0f, Ef = 0.0f;
+            if (wkey > kOrdNegInf) {                          // (warp-uniform) the segment holds a finite logit
+                const float fmx = bf16_bits_to_float(ord16_inv(wkey));
+                Ef = rintf(fminf(fmaxf(fmaf(fmx, c32, 1.0f), -1e9f), 1e9f));
+                const float nE = -Ef;
+                float s0 = 0.0f, s1 = 0.0f;
 #pragma unroll
-            for (int e8 = 0; e8 < 8; ++e8) {
-                const uint32_t bits = (e8 & 1) ? (ww[e8 >> 1] >> 16) : (ww[e8 >> 1] & 0xFFFFu);
-                const double e = exp(((double)bf16_bits_to_float(bits) - m) / tau);
-                mine += e;
-                if (e > 0.0) live = v8 * 8 + e8;
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t cw = max_bf16x2(ww[i], 0xF149F149u);           // -inf -> -1e30: keeps the two-step product finite
+                    const float lo = __uint_as_float(cw << 16), hi = __uint_as_float(cw & 0xFFFF0000u);
+                    s0 += ex2_approx(fmaf(lo, c_lo, fmaf(lo, c_hi, nE)));
+                    s1 += ex2_approx(fmaf(hi, c_lo, fmaf(hi, c_hi, nE)));
+                }
+                sum = s0 + s1;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
             }
+            if (lane == 0) { q.part[sg].sum = sum; q.part[sg].E = (int)Ef; }
         }
-    } else {
-        for (int v = lo; v < hi; ++v) {
-            const double e = exp(((double)logit(v) - m) / tau);
-            mine += e;
-            if (e > 0.0) live = v;
-        }
-    }
-    (void)inv_tau;
-    double incl = mine;
+        __syncthreads();
+        int e = -0x7FFFFFFF;
+        for (int sg = tid; sg < nseg; sg += kVerifyThreads) if (q.part[sg].sum > 0.0f) e = max(e, q.part[sg].E);
+        e = __reduce_max_sync(0xFFFFFFFFu, e);
+        if (lane == 0) q.wE[wp] = e;
+        __syncthreads();
+        int Eg = q.wE[0];
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const double up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += up;
-    }
-    if (lane == 31) q.wsum[wp] = incl;
-    __syncthreads();
-    double before = 0.0, S = 0.0;
+        for (int i = 1; i < kVerifyThreads / 32; ++i) Eg = max(Eg, q.wE[i]);
+        fast = Eg > -kSampleExpLimit && Eg < kSampleExpLimit;                     // the same for every thread
+        if (fast) {
+            if (wp == 0) {                                    // running sums over the segments, in token order
+                double carry = 0.0;
+                for (int s0 = 0; s0 < nseg; s0 += 32) {
+                    const int sg = s0 + lane;
+                    double v = 0.0;
+                    if (sg < nseg) { const SegPart pt = q.part[sg]; v = pt.sum > 0.0f ? ldexp((double)pt.sum, pt.E - Eg) : 0.0; }
+                    double incl = v;
 #pragma unroll
-    for (int i = 0; i < kVerifyThreads / 32; ++i) { const double x = q.wsum[i]; S += x; before += i < wp ? x : 0.0; }
-    incl += before;
-    const double excl = incl - mine;
-    const double t = uniform53(seed, step, b, j) * S;
-    atomicMax(&q.last_live, live);
-    if (incl > t && !(excl > t) && hi > lo) {                // the stretch in which the running sum passes t
-        double run = excl;
-        int y = live;
-        for (int v = lo; v < hi; ++v) {
-            run += exp(((double)logit(v) - m) / tau);
-            if (run > t) { y = v; break; }
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const double up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                        if (lane >= o) incl += up;
+                    }
+                    incl += carry;
+                    __syncwarp();
+                    if (sg < nseg) q.cum[sg] = incl;
+                    carry = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                }
+                if (lane == 0) q.S = carry;
+            }
+            __syncthreads();
+            const double t = u * q.S;
+            for (int sg = tid; sg < nseg; sg += kVerifyThreads) {
+                const double c = q.cum[sg];
+                if (c > t) atomicMin(&q.seg, sg);
+                if (c > (sg > 0 ? q.cum[sg - 1] : 0.0)) atomicMax(&q.live_seg, sg);
+            }
+            __syncthreads();
+            int sg = q.seg;
+            if (sg == 0x7FFFFFFF) sg = q.live_seg < 0 ? 0 : q.live_seg;          // u*S rounded up to S: the last segment with a positive sum
+            const double before = sg > 0 ? q.cum[sg - 1] : 0.0;
+            // inside the segment: four logits per thread, double precision
+            const int t0 = sg * kSegTokens + 4 * tid;
+            double ev[4] = {0.0, 0.0, 0.0, 0.0};
+            int live = -1;
+            if (t0 < p.V) {                                   // V is a multiple of 8, so all four exist
+                const uint2 x = *reinterpret_cast<const uint2*>(row + t0);
+                const uint32_t h[4] = {x.x & 0xFFFFu, x.x >> 16, x.y & 0xFFFFu, x.y >> 16};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float xf = bf16_bits_to_float(h[i]);
+                    ev[i] = xf == -INFINITY ? 0.0 : exp2((double)xf * c64 - (double)Eg);
+                    if (ev[i] > 0.0) live = t0 + i;
+                }
+            }
+            const double mine = ((ev[0] + ev[1]) + ev[2]) + ev[3];
+            double incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            if (lane == 31) q.wsum[wp] = incl;
+            __syncthreads();
+            double base = before;                             // running sum where this warp's stretch begins (one fixed order)
+            for (int i = 0; i < wp; ++i) base += q.wsum[i];
+            double prev = __shfl_up_sync(0xFFFFFFFFu, incl, 1);
+            if (lane == 0) prev = 0.0;
+            const double excl_t = base + prev, incl_t = base + incl;
+            atomicMax(&q.last_live, live);
+            if (incl_t > t && !(excl_t > t)) {                // this thread's four logits: one thread
+                double run = excl_t;
+                int yy = live;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    run += ev[i];
+                    if (run > t && ev[i] > 0.0) { yy = t0 + i; break; }
+                }
+                atomicMax(&q.chosen, yy);
+            }
+            __syncthreads();
+            y = q.chosen;
+            if (y < 0) y = q.last_live < 0 ? min(sg * kSegTokens, p.V - 1) : q.last_live;   // the exact sums end just below u*S: the segment's last live token
         }
-        atomicMax(&q.chosen, y);                             // (at most one thread gets here)
     }
-    __syncthreads();
-    int y = q.chosen;
-    if (y < 0) y = q.last_live < 0 ? 0 : q.last_live;        // rounding left no stretch: the last token with a positive term
+    if (!fast) y = sample_row_plain(q, row, p.V, p.aligned != 0, tau, u);
     verify_tail(s, w, p, b, j, ns, y, tok, par, accept_len, accept_tokens, accept_nodes, next_root);
 }
 

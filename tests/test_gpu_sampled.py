@@ -10,7 +10,8 @@ from paper_2406_17276_b200 import binding, synth
 from tests._gpu import dev_table, poisoned_verify_out, record_parity
 
 pytestmark = pytest.mark.gpu
-MARGIN = 1e-11        # a draw may fall the other way only where u*S sits this close (relative to S) to a running sum
+MARGIN = 2e-6         # a draw may fall the other way only where u*S sits this close (relative to S) to a running sum:
+                      # the library adds up each 512-logit segment in single precision (a few 1e-7 of S at worst)
 
 
 def _run(w, taus, H=None, V=None, steps=2, test_id=None):

@@ -72,6 +72,41 @@ def test_node_budgets_beyond_256(request, n, k, D, B):
     assert t["exact"] > 0 and t["near_tie"] + t["stop_near_tie"] <= 0.05 * (t["exact"] + 1)
 
 
+@pytest.mark.parametrize("name,V,H,steps,delta", [("c4", 20000, 512, 25, NEG_INF), ("c2", 20000, 512, 60, 0.2), ("c1", 32000, 4096, 100, NEG_INF)])
+def test_free_running_chain_leaves_the_oracle_only_at_a_near_tie(request, name, V, H, steps, delta):
+    """The library decodes on its own: every step starts from the token its own verification accepted last
+    (Algorithm 2's Concat).  The oracle runs its own chain from the same first roots.  As long as a sequence
+    has agreed in every earlier step both sides see the same root; the first step whose integer outputs differ
+    must be one where the oracle reports a selection boundary closer than 1e-6 (or a loop test within
+    tolerance), and such sequences are counted."""
+    w = synth.WORKLOADS[name]
+    ld, lt = synth.make_tables(w, H=H, V=V)
+    ot = binding.OptTree(V, H, w.n, w.k, w.max_depth, w.batch)
+    d_ld, d_lt = dev_table(ld), dev_table(lt)
+    memo = oracle.Memo(w.k, cap=4 * H)
+    g_roots = synth.root_tokens(w.batch, V, w.seed + 3)
+    o_roots = g_roots.copy()
+    in_sync = np.ones(w.batch, bool)
+    st = new_totals()
+    for _ in range(steps):
+        g = gpu_step(ot, d_ld, d_lt, g_roots, delta)
+        o = oracle.table_step(ld, lt, o_roots, w.n, w.k, w.max_depth, float(np.float32(delta)), memo=memo)
+        for b in np.nonzero(in_sync)[0]:
+            assert g_roots[b] == o_roots[b]
+            ob = _compare._slice(o, b)
+            if _compare._ints_equal(g, ob, b, True):
+                st["exact"] += 1
+                _compare._check_floats(g, ob, b, st)
+            else:
+                near = o.min_gap[b] < _compare.GAP_EXEMPT or o.stop_margin[b] < _compare.FLOAT_RTOL * max(1.0, o.expected_len[b])
+                assert near, f"sequence {b} left the oracle's chain at a step whose smallest gap is {o.min_gap[b]:.3e}"
+                st["near_tie"] += 1
+                in_sync[b] = False
+        g_roots, o_roots = g["next_root"].copy(), o.next_root.copy()
+    record_parity(request.node.nodeid, st)
+    assert in_sync.sum() >= 0.9 * w.batch
+
+
 def test_two_runs_are_bit_identical():
     w = synth.WORKLOADS["c4"]
     ld, lt = synth.make_tables(w, H=256, V=20000)

@@ -48,6 +48,7 @@ def test_study_agrees_with_host_side_definitions():
             assert np.array_equal(first["roots"][s + 1], o.next_root) or np.any(o.min_gap < 1e-6)
     sh = res["shapes"]
     assert sh["opt_tree"]["mean_expected_length_plus_1"] >= sh["binary"]["mean_expected_length_plus_1"] - 1e-9
-    assert sh["opt_tree"]["mean_expected_length_plus_1"] >= sh["sequence"]["mean_expected_length_plus_1"] - 1e-9
+    assert sh["opt_tree"]["mean_expected_length_plus_1"] >= sh["4-ary"]["mean_expected_length_plus_1"] - 1e-9
+    # (the sequence draft may go deeper than the adaptive tree's depth limit, so no such bound holds for it)
     h = np.array(res["hist_rows_rounded_EA_plus_1_cols_A"])
     assert h.sum() == steps * w.batch
