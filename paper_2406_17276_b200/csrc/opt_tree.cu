@@ -272,7 +272,8 @@ struct BuildSink {
     }
     // pick != null (pruned draft): only the layer slots pick[0..nl) are sent out, as frontier rows 0..nl;
     // the map from frontier row to layer slot is left in fmap for the next selection.
-    __device__ void publish_layer(LayerScratch& ls, int b, int d, int nl, unsigned g0, const int* pick = nullptr,
+    template <class LS>
+    __device__ void publish_layer(LS& ls, int b, int d, int nl, unsigned g0, const int* pick = nullptr,
                                   int32_t* fmap = nullptr) {
         const int lane = threadIdx.x & 31;
         g0 = __shfl_sync(0xFFFFFFFFu, g0, 0);
@@ -310,7 +311,8 @@ struct BuildSink {
     }
     // Pruned draft, a whole layer job with one selection (see select_running_team).  Returns the number
     // of rows of the next layer, or -1 if the sequence is finished.
-    __device__ int merged_layer_job(LayerScratch& ls, const SeqWork& sw, int b, int d, int fsize, int nR_old, int off) {
+    template <class LS>
+    __device__ int merged_layer_job(LS& ls, const SeqWork& sw, int b, int d, int fsize, int nR_old, int off) {
         const int lane = threadIdx.x & 31;
         const int nvalid = fsize * p.kk, reserve = nvalid < p.n ? nvalid : p.n;
         stage_layer_candidates(ls, sw, fsize, p.k, off);
@@ -375,13 +377,15 @@ struct BuildSink {
     // The layer warp follows its sequences (layer_follow); whenever a layer is complete it hands the
     // selection to the whole team: the job goes into shared memory, the team barrier starts it.  The
     // assistants wait at that barrier in between and leave when they find a job of kind 0.
-    __device__ void layer_loop(LayerScratch& ls) {
+    template <class LS>
+    __device__ void layer_loop(LS& ls) {
         layer_follow(ls);
         if ((threadIdx.x & 31) == 0) ls.job.kind = 0;
         __syncwarp();
         team_sync();
     }
-    __device__ void layer_assist(LayerScratch& ls, int tw) {
+    template <class LS>
+    __device__ void layer_assist(LS& ls, int tw) {
         const int tt = tw * 32 + (int)(threadIdx.x & 31);
         for (;;) {
             team_sync();
@@ -392,7 +396,8 @@ struct BuildSink {
             else select_layer_team_big<kPrune>(ls, j, tt, w.status);
         }
     }
-    __device__ void layer_follow(LayerScratch& ls) {
+    template <class LS>
+    __device__ void layer_follow(LS& ls) {
         const int lane = threadIdx.x & 31;
         constexpr int kOwn = 4;                            // sequences one layer warp follows at a time
         for (int b0 = blockIdx.x; b0 < p.B; b0 += kOwn * gridDim.x) {
@@ -513,14 +518,14 @@ struct BuildSink {
 
 // Algorithm 1 for a whole batch in one launch: persistent CTAs take rows from their mailboxes; layers
 // of different sequences overlap freely because sequences never exchange data.
-template <bool kPrune>
+template <bool kPrune, int NCAP>
 __global__ void __launch_bounds__(kThreads)
 build_kernel(Workspace w, Params p, const uint16_t* __restrict__ draft, opt_tree_out out) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
+    CtaSmemT<NCAP>& s = *reinterpret_cast<CtaSmemT<NCAP>*>(smem_raw);
     BuildSource<kPrune> src{w, p, draft};
     BuildSink<kPrune> sink{w, p, out};
-    run_pipeline(s, src, sink, p.V, p.k, p.n, p.aligned != 0, w.status);
+    run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, w.status);
 }
 
 // The row step alone over a list of rows (static round-robin over the CTAs).
@@ -540,8 +545,8 @@ struct ListSource {
 };
 struct ListSink {
     int32_t* tok_out; double* prob_out; int k;
-    __device__ void layer_loop(LayerScratch&) {}
-    __device__ void layer_assist(LayerScratch&, int) {}
+    template <class LS> __device__ void layer_loop(LS&) {}
+    template <class LS> __device__ void layer_assist(LS&, int) {}
     __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch&) {
         const int lane = threadIdx.x & 31;
         if (lane < k) {
@@ -557,7 +562,7 @@ row_topk_kernel(Params p, const uint16_t* __restrict__ logits, const int32_t* __
     CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
     ListSource src{logits, rows, nrows, p.V, p.H, (int)blockIdx.x, (int)gridDim.x, status};
     ListSink sink{tok_out, prob_out, p.k};
-    run_pipeline(s, src, sink, p.V, p.k, p.n, p.aligned != 0, status);
+    run_pipeline(s, src, sink, p.V, p.k, p.aligned != 0, status);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -578,12 +583,12 @@ __global__ void layers_begin_kernel(Workspace w, Params p) {
     w.fmap[(size_t)b * p.n] = 0;
 }
 
+template <int NCAP>
 __global__ void __launch_bounds__(kTeam)
 layer_step_kernel(Workspace w, Params p, int fstride, opt_tree_out out, int32_t* next_tokens, int32_t* next_parent,
                   int32_t* next_count) {
-    __shared__ LayerScratch ls;
-    extern __shared__ __align__(16) unsigned char ls_tail[];       // the n-sized arrays (layer_tail_bytes(n))
-    if (threadIdx.x == 0) layer_tail_carve(ls, ls_tail, p.n);
+    extern __shared__ __align__(16) unsigned char ls_raw[];
+    LayerScratchT<NCAP>& ls = *reinterpret_cast<LayerScratchT<NCAP>*>(ls_raw);
     grid_dependency_wait();
     const int b = blockIdx.x, tt = threadIdx.x, lane = tt & 31;
     for (int i = tt; i < 3 * 256; i += kTeam) (&ls.thist[0][0])[i] = 0;
@@ -1101,19 +1106,19 @@ __global__ void __launch_bounds__(kThreads)
 wait_probe_kernel(int* result, const unsigned long long* zero_words, long long limit, int polls) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CtaSmem& s = *reinterpret_cast<CtaSmem*>(smem_raw);
-    pipeline_init(s, 1);
+    pipeline_init(s.core, s.layer);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp == 0) {
-        mbar_wait_warp(&s.full_bar[0], 0u, &result[0], limit);
+        mbar_wait_warp(&s.core.full_bar[0], 0u, &result[0], limit);
     } else if (warp == 1) {
-        if (lane == 0) mbar_wait_thread(&s.full_bar[1], 0u, &result[1], limit);
+        if (lane == 0) mbar_wait_thread(&s.core.full_bar[1], 0u, &result[1], limit);
     } else if (warp == 2) {
         if (lane == 0) poll_phat_word(zero_words, &result[2], polls);
     } else if (warp == 3) {
         if (lane == 0) poll_tok_word(reinterpret_cast<const unsigned int*>(zero_words + 1), &result[3], polls);
     } else if (warp == 4) {
         NeverSource src;
-        fetcher_role(s, src, &result[4], limit);
+        fetcher_role(s.core, src, &result[4], limit);
     }
 }
 
@@ -1188,19 +1193,25 @@ extern "C" {
 
 // CTAs of the persistent kernels on the current device (one CTA of kThreads per SM as long as its
 // shared memory fits); 0 if there is no usable device.
-// Shared memory of a CTA of the persistent kernels for node budget n: the fixed part and the layer team's
-// n-sized arrays behind it.
-static size_t cta_smem_bytes(int n) { return sizeof(ot::CtaSmem) + ((ot::layer_tail_bytes(n) + 15) & ~(size_t)15); }
+// Shared memory of a CTA of the persistent kernels for node budget n (one of two layouts).
+static bool small_n(int n) { return n <= ot::kSmallN; }
+static size_t cta_smem_bytes(int n) { return small_n(n) ? sizeof(ot::CtaSmemT<ot::kSmallN>) : sizeof(ot::CtaSmemT<ot::kMaxN>); }
+static size_t layer_smem_bytes(int n) { return small_n(n) ? sizeof(ot::LayerScratchT<ot::kSmallN>) : sizeof(ot::LayerScratchT<ot::kMaxN>); }
 
 static int persistent_grid(int n) {
     int dev = 0, per_sm = 0, sms = 0;
-    const int most = (int)cta_smem_bytes(OPT_TREE_MAX_N);
+    constexpr int S = ot::kSmallN, L = ot::kMaxN;
+    const auto dyn = cudaFuncAttributeMaxDynamicSharedMemorySize;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
-    if (cudaFuncSetAttribute(ot::build_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-        cudaFuncSetAttribute(ot::build_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-        cudaFuncSetAttribute(ot::row_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-        cudaFuncSetAttribute(ot::layer_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ot::layer_tail_bytes(OPT_TREE_MAX_N)) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ot::build_kernel<true>, ot::kThreads, cta_smem_bytes(n)) != cudaSuccess ||
+    if (cudaFuncSetAttribute(ot::build_kernel<false, S>, dyn, (int)sizeof(ot::CtaSmemT<S>)) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::build_kernel<true, S>, dyn, (int)sizeof(ot::CtaSmemT<S>)) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::build_kernel<false, L>, dyn, (int)sizeof(ot::CtaSmemT<L>)) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::build_kernel<true, L>, dyn, (int)sizeof(ot::CtaSmemT<L>)) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::row_topk_kernel, dyn, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::layer_step_kernel<S>, dyn, (int)sizeof(ot::LayerScratchT<S>)) != cudaSuccess ||
+        cudaFuncSetAttribute(ot::layer_step_kernel<L>, dyn, (int)sizeof(ot::LayerScratchT<L>)) != cudaSuccess ||
+        (small_n(n) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ot::build_kernel<true, S>, ot::kThreads, sizeof(ot::CtaSmemT<S>))
+                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ot::build_kernel<true, L>, ot::kThreads, sizeof(ot::CtaSmemT<L>))) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
         cudaGetLastError();
         return 0;
@@ -1271,12 +1282,9 @@ static int build_common(opt_tree_ctx* ctx, const void* draft, const int32_t* roo
     p.prune = prune;
     const long long init_threads = (long long)ctx->grid * ctx->mcap > B ? (long long)ctx->grid * ctx->mcap : B;
     launch_after(ot::init_build_kernel, dim3((unsigned)((init_threads + 255) / 256)), dim3(256), 0, st, ctx->ws, p, root_token);
-    if (prune)
-        launch_after(ot::build_kernel<true>, dim3(ctx->grid), dim3(ot::kThreads), ctx->smem, st,
-                     ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
-    else
-        launch_after(ot::build_kernel<false>, dim3(ctx->grid), dim3(ot::kThreads), ctx->smem, st,
-                     ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
+    auto kernel = small_n(ctx->cfg.n) ? (prune ? ot::build_kernel<true, ot::kSmallN> : ot::build_kernel<false, ot::kSmallN>)
+                                      : (prune ? ot::build_kernel<true, ot::kMaxN> : ot::build_kernel<false, ot::kMaxN>);
+    launch_after(kernel, dim3(ctx->grid), dim3(ot::kThreads), ctx->smem, st, ctx->ws, p, static_cast<const uint16_t*>(draft), *out);
     ctx->launches += 2;
     int rc = check_launch();
     if (rc == OPT_TREE_OK && rows_read &&
@@ -1365,10 +1373,11 @@ int opt_tree_layers_step(opt_tree_ctx* ctx, const void* frontier_logits, int32_t
     ot::Params pr = p;
     pr.H = nrows;                                            // the dense buffer is the "table" of the row step
     const int grid = nrows < ctx->grid ? nrows : ctx->grid;
-    launch_after(ot::row_topk_kernel, dim3(grid), dim3(ot::kThreads), ctx->smem, st,
+    launch_after(ot::row_topk_kernel, dim3(grid), dim3(ot::kThreads), sizeof(ot::CtaSmem), st,
                  pr, static_cast<const uint16_t*>(frontier_logits), static_cast<const int32_t*>(nullptr), nrows, ctx->ws.rtok,
                  ctx->ws.rprob, ctx->ws.status);
-    launch_after(ot::layer_step_kernel, dim3(B), dim3(ot::kTeam), ot::layer_tail_bytes(ctx->cfg.n), st, ctx->ws, p, frontier_stride, *out, next_tokens,
+    launch_after(small_n(ctx->cfg.n) ? ot::layer_step_kernel<ot::kSmallN> : ot::layer_step_kernel<ot::kMaxN>, dim3(B), dim3(ot::kTeam),
+                 layer_smem_bytes(ctx->cfg.n), st, ctx->ws, p, frontier_stride, *out, next_tokens,
                  next_parent, next_count);
     ctx->launches += 2;
     return check_launch();
@@ -1380,7 +1389,7 @@ int opt_tree_row_softmax_topk(opt_tree_ctx* ctx, const void* logits, const int32
     if (nrows == 0) return OPT_TREE_OK;
     const ot::Params p = make_params(ctx, logits, 0.0f);
     const int grid = nrows < ctx->grid ? nrows : ctx->grid;
-    ot::row_topk_kernel<<<grid, ot::kThreads, ctx->smem, static_cast<cudaStream_t>(stream)>>>(
+    ot::row_topk_kernel<<<grid, ot::kThreads, sizeof(ot::CtaSmem), static_cast<cudaStream_t>(stream)>>>(
         p, static_cast<const uint16_t*>(logits), rows, nrows, tok_out, prob_out, ctx->ws.status);
     ctx->launches++;
     return check_launch();
@@ -1422,13 +1431,13 @@ int opt_tree_step_host(opt_tree_ctx* ctx, const void* draft, const void* target,
 int opt_tree_selftest_waits(opt_tree_ctx* ctx, int32_t* result, void* stream) {
     if (!ctx || !result) return OPT_TREE_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaFuncSetAttribute(ot::wait_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cta_smem_bytes(1)) != cudaSuccess ||
+    if (cudaFuncSetAttribute(ot::wait_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ot::CtaSmem)) != cudaSuccess ||
         cudaMemsetAsync(result, 0, OPT_TREE_SELFTEST_WAITS * sizeof(int32_t), st) != cudaSuccess ||
         cudaMemsetAsync(ctx->ws.rprob, 0, 2 * sizeof(unsigned long long), st) != cudaSuccess) {     // two words nobody writes
         cudaGetLastError();
         return OPT_TREE_ERR_CUDA;
     }
-    ot::wait_probe_kernel<<<1, ot::kThreads, cta_smem_bytes(1), st>>>(
+    ot::wait_probe_kernel<<<1, ot::kThreads, sizeof(ot::CtaSmem), st>>>(
         result, reinterpret_cast<const unsigned long long*>(ctx->ws.rprob), 1ll << 16, 1 << 10);
     ctx->launches++;
     return check_launch();

@@ -28,18 +28,17 @@
 
 namespace ot {
 
-// n: the context's node budget; the layer team's n-sized arrays start right behind the CtaSmem.
-__device__ __forceinline__ void pipeline_init(CtaSmem& s, int n) {
+template <class LS>
+__device__ __forceinline__ void pipeline_init(CtaCore& s, LS& layer) {
     if (threadIdx.x == 0) {
-        layer_tail_carve(s.layer, reinterpret_cast<unsigned char*>(&s) + sizeof(CtaSmem), n);
         for (int i = 0; i < kStages; ++i) { mbar_init(&s.full_bar[i], 1); mbar_init(&s.empty_bar[i], kConsumerWarps); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(&s.ready_bar[i], kConsumerWarps); mbar_init(&s.free_bar[i], 1); }
         for (int i = 0; i < kDesc; ++i) { mbar_init(&s.desc_full[i], 1); mbar_init(&s.desc_empty[i], kConsumerWarps); }
         s.stop_row = 0x7FFFFFFF;
         mbar_fence_init();
     }
-    for (int i = threadIdx.x; i < 3 * 256; i += kThreads) (&s.layer.thist[0][0])[i] = 0;
-    if (threadIdx.x == 0) { s.layer.cache_b = -1; s.layer.cache_d = -1; }
+    for (int i = threadIdx.x; i < 3 * 256; i += kThreads) (&layer.thist[0][0])[i] = 0;
+    if (threadIdx.x == 0) { layer.cache_b = -1; layer.cache_d = -1; }
     __syncthreads();
 }
 
@@ -56,7 +55,7 @@ __device__ __forceinline__ void pipeline_init(CtaSmem& s, int n) {
 // Once a Source has said "no more work" no ticket of this CTA can still turn into a row.
 constexpr int kFetchLanes = 4;
 template <class Source>
-__device__ void fetcher_role(CtaSmem& s, Source& src, int* status, long long limit = kWaitCycles) {
+__device__ void fetcher_role(CtaCore& s, Source& src, int* status, long long limit = kWaitCycles) {
     const int lane = threadIdx.x & 31;
     const unsigned below = (1u << lane) - 1u;
     bool holding = false;                 // this lane has a ticket
@@ -119,7 +118,7 @@ __device__ __noinline__ void copy_chunk_plain(uint16_t* stage, const uint16_t* s
 
 // With `aligned` false (table base or row pitch not 16-byte aligned) the whole warp copies the
 // chunk with ordinary loads instead of a bulk copy.
-__device__ void issuer_role(CtaSmem& s, int V, bool aligned, int* status) {
+__device__ void issuer_role(CtaCore& s, int V, bool aligned, int* status) {
     const int lane = threadIdx.x & 31;
     const int nchunks = (V + kChunkElems - 1) / kChunkElems;
     long long g = 0;
@@ -154,7 +153,7 @@ __device__ void issuer_role(CtaSmem& s, int V, bool aligned, int* status) {
 // A warp takes its share of a chunk out of the ring into registers and hands the stage back at once
 // (so the issuer can refill it while the exponentials run); a row's descriptor is only looked at for
 // its stop flag.
-__device__ void consumer_role(CtaSmem& s, int cwarp, int V, int* status) {
+__device__ void consumer_role(CtaCore& s, int cwarp, int V, int* status) {
     const int lane = threadIdx.x & 31, tid = cwarp * 32 + lane;     // index among the consumer threads
     const int nchunks = (V + kChunkElems - 1) / kChunkElems;
     ThreadAcc acc;
@@ -193,7 +192,7 @@ __device__ void consumer_role(CtaSmem& s, int cwarp, int V, int* status) {
 // ---- finisher warps ----------------------------------------------------------------------------
 // Sink::row_done(const RowDesc&, const RowOut&, FinScratch&) is called by the whole warp.
 template <class Sink>
-__device__ void finisher_role(CtaSmem& s, Sink& sink, int fidx, int V, int k, bool aligned, int* status) {
+__device__ void finisher_role(CtaCore& s, Sink& sink, int fidx, int V, int k, bool aligned, int* status) {
     const int lane = threadIdx.x & 31;
     FinScratch& f = s.fin[fidx];
     for (int r = fidx;; r += kFinishers) {
@@ -223,17 +222,18 @@ __device__ void finisher_role(CtaSmem& s, Sink& sink, int fidx, int V, int k, bo
     }
 }
 
-template <class Source, class Sink>
-__device__ __forceinline__ void run_pipeline(CtaSmem& s, Source& src, Sink& sink, int V, int k, int n, bool aligned, int* status) {
-    pipeline_init(s, n);
+template <class Smem, class Source, class Sink>
+__device__ __forceinline__ void run_pipeline(Smem& sm, Source& src, Sink& sink, int V, int k, bool aligned, int* status) {
+    CtaCore& s = sm.core;
+    pipeline_init(s, sm.layer);
     grid_dependency_wait();                                // shared memory is set up; global memory from here on
     const int warp = threadIdx.x >> 5;
     if (warp < kConsumerWarps) { consumer_role(s, warp, V, status); return; }
     const int helper = warp - kConsumerWarps;
     if (helper == kHelperIssuer) issuer_role(s, V, aligned, status);
     else if (helper == kHelperFetcher) fetcher_role(s, src, status);
-    else if (helper == kHelperLayer) sink.layer_loop(s.layer);
-    else if (helper < kHelperFirstFinisher) sink.layer_assist(s.layer, helper - kHelperLayer);
+    else if (helper == kHelperLayer) sink.layer_loop(sm.layer);
+    else if (helper < kHelperFirstFinisher) sink.layer_assist(sm.layer, helper - kHelperLayer);
     else finisher_role(s, sink, helper - kHelperFirstFinisher, V, k, aligned, status);
 }
 

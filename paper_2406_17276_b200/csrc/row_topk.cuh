@@ -81,18 +81,21 @@ struct LayerJob {                  // what the layer warp hands its assistants (
 };
 
 constexpr int kStageCap = 1024;                    // candidates of a layer that the shared-memory staging holds
+constexpr int kSmallN = 256;                       // node budgets up to this use the smaller of the two scratch layouts
 
-// Private to the layer team of a CTA.  The arrays whose length follows the node budget n are not
-// members: they live behind the CTA's fixed shared memory, sized by the context's n (see
-// layer_tail_bytes / layer_tail_carve), so that a small n keeps the CTA's shared memory small.
-struct alignas(16) LayerScratch {
-    unsigned long long* keys;                  // [max(kStageCap, 2n) + 2] staged candidate keys, then the keys of R + layer
-    unsigned long long* lkeys;                 // [n]  keys of the new layer, slot order
-    double* vals;                              // [n]  path values of the new running top-n
-    int* gids;                                 // [2n]
-    int* rsel;                                 // [n]  gids of the new running top-n, ascending
-    int* ltok;                                 // [n]  tokens of the new layer, slot order
+// Private to the layer team of a CTA.  NCAP is the largest node budget the layout serves: the kernels
+// exist once for NCAP = kSmallN and once for NCAP = kMaxN, so that the common small budgets keep the
+// CTA's shared memory (and with it the SM's L1) where it is best for them.
+template <int NCAP>
+struct alignas(16) LayerScratchT {
+    static constexpr int kKeys = (2 * NCAP > kStageCap ? 2 * NCAP : kStageCap) + 2;
+    unsigned long long keys[kKeys];            // staged candidate keys, then the keys of R + layer
+    unsigned long long lkeys[NCAP];            // keys of the new layer, slot order
+    double vals[NCAP];                         // path values of the new running top-n
     int toks[kStageCap + 4];                   // staged candidate tokens
+    int gids[2 * NCAP];
+    int rsel[NCAP];                            // gids of the new running top-n, ascending
+    int ltok[NCAP];                            // tokens of the new layer, slot order
     int hist[256];
     int thist[3][256];                         // the team's digit counts, rotating (all zero between selections)
     unsigned long long red_or[kTeamWarps], red_and[kTeamWarps];
@@ -109,11 +112,11 @@ static_assert(sizeof(FinScratch) % 16 == 0 && offsetof(FinScratch, hist) % 16 ==
 // rows between "descriptor written" and "finisher has its copy": kDesc known + 1 streaming + kSlots handed on
 static_assert(kDescRing >= kDesc + 1 + kSlots + 1, "descriptor ring too short");
 
-struct alignas(128) CtaSmem {
+// The row pipeline's part of a CTA's shared memory (the same for every node budget) ...
+struct alignas(128) CtaCore {
     uint16_t stage[kStages][kChunkElems];
     RowSlot slot[kSlots];
     FinScratch fin[kFinishers];
-    LayerScratch layer;
     RowDesc desc[kDescRing];                   // row r in entry r % kDescRing
     unsigned long long full_bar[kStages];      // issuer -> consumers (bulk copy landed)
     unsigned long long empty_bar[kStages];     // consumers -> issuer (stage may be overwritten)
@@ -123,21 +126,14 @@ struct alignas(128) CtaSmem {
     unsigned long long desc_empty[kDesc];      // consumers -> fetcher (descriptor may be overwritten)
     volatile int stop_row;                     // first row index that is the stop marker
 };
-
-// Bytes of the n-sized arrays of LayerScratch, and their placement behind `base` (16-byte aligned).
-__host__ __device__ inline size_t layer_tail_bytes(int n) {
-    const size_t nk = (size_t)(2 * n > kStageCap ? 2 * n : kStageCap) + 2;
-    return nk * 8 + (size_t)n * 8 * 2 + (size_t)n * 4 * 4;
-}
-__device__ __forceinline__ void layer_tail_carve(LayerScratch& s, unsigned char* base, int n) {
-    const size_t nk = (size_t)(2 * n > kStageCap ? 2 * n : kStageCap) + 2;
-    s.keys = reinterpret_cast<unsigned long long*>(base);
-    s.lkeys = s.keys + nk;
-    s.vals = reinterpret_cast<double*>(s.lkeys + n);
-    s.gids = reinterpret_cast<int*>(s.vals + n);
-    s.rsel = s.gids + 2 * n;
-    s.ltok = s.rsel + n;
-}
+// ... and the whole of it, with the layer team's scratch.
+template <int NCAP>
+struct alignas(128) CtaSmemT {
+    CtaCore core;
+    LayerScratchT<NCAP> layer;
+};
+using CtaSmem = CtaSmemT<kSmallN>;
+static_assert(sizeof(CtaSmemT<kMaxN>) <= 232448, "the larger layout must fit a CTA's shared memory");
 
 __device__ __forceinline__ int chunk_elems(int V, int c) {
     int rem = V - c * kChunkElems;

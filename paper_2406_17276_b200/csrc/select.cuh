@@ -133,7 +133,8 @@ struct TreeOut {           // mirrors opt_tree_out, pointers offset to the seque
 // Starts the asynchronous copies of a layer's candidates (path values and tokens) into the layer
 // warp's scratch; the layer warp waits for them before it starts the team.  Separate so that other round trips (the
 // mailbox reservations) can be in flight at the same time.
-__device__ __forceinline__ void stage_layer_candidates(LayerScratch& s, const SeqWork& w, int fsize, int k, int off = 0) {
+template <class LS>
+__device__ __forceinline__ void stage_layer_candidates(LS& s, const SeqWork& w, int fsize, int k, int off = 0) {
     const int lane = threadIdx.x & 31;
     const int N = fsize * k;
     if (off + N > kStageCap) return;                       // (off is even: the copies keep their 16-byte alignment)
@@ -188,8 +189,8 @@ __device__ __forceinline__ int team_excl_scan(int v, int* wtot, int tw, int& tot
 __device__ __forceinline__ unsigned long long key_of_word(unsigned long long x) {
     return x == ~0ull ? 0ull : (x & 0x7FFFFFFFFFFFFFFFull) + 1ull;
 }
-template <bool kGlobal>
-__device__ int team_radix_select(LayerScratch& s, const unsigned long long* gw, int N, int need, int tt, unsigned long long key_or,
+template <bool kGlobal, class LS>
+__device__ int team_radix_select(LS& s, const unsigned long long* gw, int N, int need, int tt, unsigned long long key_or,
                                  unsigned long long key_and, unsigned long long& thr, int& need_eq) {
     const int lane = threadIdx.x & 31;
     const unsigned long long diff = key_or ^ key_and;
@@ -267,8 +268,8 @@ __device__ int team_radix_select(LayerScratch& s, const unsigned long long* gw, 
 // The team's part of a layer selection (N = fsize * k <= 1024; the candidates were staged into s
 // by the layer warp).  On return (after a last barrier) the new layer's nodes are in T and its
 // tokens and keys in s.ltok / s.lkeys.  Returns nl.
-template <bool kPrune>
-__device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j, int tt, int* status) {
+template <bool kPrune, class LS>
+__device__ __noinline__ int select_layer_team(LS& s, const LayerJob& j, int tt, int* status) {
     const int lane = threadIdx.x & 31, tw = tt >> 5;
     const int N = j.fsize * j.k;
     const int nvalid = j.fsize * j.kk;
@@ -350,7 +351,8 @@ __device__ __noinline__ int select_layer_team(LayerScratch& s, const LayerJob& j
 // the new top-n (gids ascending; also written to j.Rnew), its new members are T's nodes
 // gid0 .. gid0+cnt in candidate order with tokens and keys in s.ltok / s.lkeys, and s.scan_c sums
 // to the number of old members kept.  Returns |new top-n|.
-__device__ __noinline__ int select_running_team(LayerScratch& s, const LayerJob& j, int tt, int* status) {
+template <class LS>
+__device__ __noinline__ int select_running_team(LS& s, const LayerJob& j, int tt, int* status) {
     const int lane = threadIdx.x & 31, tw = tt >> 5;
     const int N = j.fsize * j.k, nRo = j.nR_old, off = j.off, M = off + N;
     const int nvalid = j.fsize * j.kk;
@@ -456,8 +458,8 @@ __device__ __noinline__ int select_running_team(LayerScratch& s, const LayerJob&
 // The team's selection for layers with more candidates than the shared-memory staging holds
 // (1024 < N <= n*k): the same steps, but every sweep reads the candidate words from global memory
 // (they sit in L2), a thread's loads eight at a time.  The candidate arrays are cleared at the end.
-template <bool kPrune>
-__device__ __noinline__ int select_layer_team_big(LayerScratch& s, const LayerJob& j, int tt, int* status) {
+template <bool kPrune, class LS>
+__device__ __noinline__ int select_layer_team_big(LS& s, const LayerJob& j, int tt, int* status) {
     const int lane = threadIdx.x & 31, tw = tt >> 5;
     const int N = j.fsize * j.k;
     const int nvalid = j.fsize * j.kk;
@@ -543,7 +545,8 @@ __device__ __noinline__ int select_layer_team_big(LayerScratch& s, const LayerJo
 
 // Once per sequence, when it is finished: T_opt = the running top-n (s.rsel / s.vals, already in
 // (depth, parent's index, sibling rank) order), packed with parent indices.
-__device__ __noinline__ void pack_tree_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nR, int n, int max_depth,
+template <class LS>
+__device__ __noinline__ void pack_tree_warp(LS& s, const SeqWork& w, const TreeOut& out, int d, int nR, int n, int max_depth,
                                             double esub, int* status) {
     const int lane = threadIdx.x & 31;
     if (out.esub_trace) for (int i = d + lane; i < max_depth; i += 32) out.esub_trace[i] = 0.0;
@@ -576,7 +579,8 @@ __device__ __noinline__ void pack_tree_warp(LayerScratch& s, const SeqWork& w, c
 // the selection), the loop test of Algorithm 1, and the packed tree if the sequence is
 // finished.  All layers of a sequence are handled by the same warp, in order.  Returns true if the
 // sequence continues with layer d+1, false if it is finished (outputs written).
-__device__ __noinline__ bool update_running_warp(LayerScratch& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
+template <class LS>
+__device__ __noinline__ bool update_running_warp(LS& s, const SeqWork& w, const TreeOut& out, int d, int nl, int n, int Dcap,
                                     int max_depth, float delta, int* status) {
     const int lane = threadIdx.x & 31;
     int* hist = s.hist;
