@@ -973,34 +973,50 @@ verify_sampled_kernel(Workspace w, Params p, const uint16_t* __restrict__ target
         const float c_lo = (float)(c64 - (double)c_hi);
         const uint4* rv = reinterpret_cast<const uint4*>(row);
         if (tid == 0) { q.chosen = -1; q.last_live = -1; q.seg = 0x7FFFFFFF; q.live_seg = -1; }
+        // two segments per turn: four 16-byte loads in flight per lane
+        const unsigned long long chi2 = pack2(c_hi, c_hi), clo2 = pack2(c_lo, c_lo);
+        constexpr int kStep = kVerifyThreads / 32;
 #pragma unroll 1
-        for (int sg = wp; sg < nseg; sg += kVerifyThreads / 32) {
-            const int v0 = sg * kSegVecs + lane, v1 = v0 + 32;
+        for (int sg0 = wp; sg0 < nseg; sg0 += 2 * kStep) {
             const uint4 pad = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-            const uint4 q0 = v0 < nv ? ld_nc_v4(rv + v0) : pad, q1 = v1 < nv ? ld_nc_v4(rv + v1) : pad;
-            uint32_t ww[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
-            uint32_t m2 = ww[0];
+            uint4 qq[2][2];
 #pragma unroll
-            for (int i = 1; i < 8; ++i) m2 = max_bf16x2(m2, ww[i]);
-            const uint32_t wkey = __reduce_max_sync(0xFFFFFFFFu, max(ord16(m2 & 0xFFFFu), ord16(m2 >> 16)));
-            float sum = 0.0f, Ef = 0.0f;
-            if (wkey > kOrdNegInf) {                          // (warp-uniform) the segment holds a finite logit
-                const float fmx = bf16_bits_to_float(ord16_inv(wkey));
-                Ef = rintf(fminf(fmaxf(fmaf(fmx, c32, 1.0f), -1e9f), 1e9f));
-                const float nE = -Ef;
-                float s0 = 0.0f, s1 = 0.0f;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const uint32_t cw = max_bf16x2(ww[i], 0xF149F149u);           // -inf -> -1e30: keeps the two-step product finite
-                    const float lo = __uint_as_float(cw << 16), hi = __uint_as_float(cw & 0xFFFF0000u);
-                    s0 += ex2_approx(fmaf(lo, c_lo, fmaf(lo, c_hi, nE)));
-                    s1 += ex2_approx(fmaf(hi, c_lo, fmaf(hi, c_hi, nE)));
-                }
-                sum = s0 + s1;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+            for (int h = 0; h < 2; ++h) {
+                const int v0 = (sg0 + h * kStep) * kSegVecs + lane, v1 = v0 + 32;
+                qq[h][0] = v0 < nv ? ld_nc_v4(rv + v0) : pad;
+                qq[h][1] = v1 < nv ? ld_nc_v4(rv + v1) : pad;
             }
-            if (lane == 0) { q.part[sg].sum = sum; q.part[sg].E = (int)Ef; }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int sg = sg0 + h * kStep;
+                if (sg >= nseg) break;                            // (warp-uniform)
+                const uint32_t ww[8] = {qq[h][0].x, qq[h][0].y, qq[h][0].z, qq[h][0].w, qq[h][1].x, qq[h][1].y, qq[h][1].z, qq[h][1].w};
+                uint32_t m2 = ww[0];
+#pragma unroll
+                for (int i = 1; i < 8; ++i) m2 = max_bf16x2(m2, ww[i]);
+                const uint32_t wkey = __reduce_max_sync(0xFFFFFFFFu, max(ord16(m2 & 0xFFFFu), ord16(m2 >> 16)));
+                float sum = 0.0f, Ef = 0.0f;
+                if (wkey > kOrdNegInf) {                          // (warp-uniform) the segment holds a finite logit
+                    const float fmx = bf16_bits_to_float(ord16_inv(wkey));
+                    Ef = rintf(fminf(fmaxf(fmaf(fmx, c32, 1.0f), -1e9f), 1e9f));
+                    const unsigned long long nE2 = pack2(-Ef, -Ef);
+                    unsigned long long acc2 = 0ull;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t cw = max_bf16x2(ww[i], 0xF149F149u);       // -inf -> -1e30: keeps the two-step product finite
+                        const unsigned long long x2 = pack2(__uint_as_float(cw << 16), __uint_as_float(cw & 0xFFFF0000u));
+                        float a0, a1;
+                        unpack2(fma2(x2, clo2, fma2(x2, chi2, nE2)), a0, a1);
+                        acc2 = add2(acc2, pack2(ex2_approx(a0), ex2_approx(a1)));
+                    }
+                    float s0, s1;
+                    unpack2(acc2, s0, s1);
+                    sum = s0 + s1;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+                }
+                if (lane == 0) { q.part[sg].sum = sum; q.part[sg].E = (int)Ef; }
+            }
         }
         __syncthreads();
         int e = -0x7FFFFFFF;
