@@ -208,7 +208,7 @@ __global__ void init_build_kernel(Workspace w, Params p, const int32_t* __restri
     for (long long j = i; j < (long long)p.B * p.n; j += (long long)gridDim.x * blockDim.x) w.fmap[j] = (int32_t)(j % p.n);
     if (i < p.B) {
         int32_t* st = w.st + (size_t)i * 8;
-        st[kStDone] = 0; st[kStNR] = 0; st[kStRows] = 0;
+        st[kStDone] = 0; st[kStNR] = 0; st[kStRows] = 0; st[kStL1] = 0;
         w.E_prev[i] = 0.0;
     }
     if (i == 0) { w.q_ctl[kQFinished] = 0; w.q_ctl[kQDone] = 0; w.q_ctl[kQCursor] = p.B; }   // the roots are rows 0 .. B-1
@@ -246,9 +246,55 @@ struct BuildSource {
 template <bool kPrune>
 struct BuildSink {
     Workspace w; Params p; opt_tree_out out;
+    // Layer 1 by the finisher of the root's row.  The root's children are the only candidates of layer 1; when
+    // they all fit the node budget nothing has to be selected: the finisher stores them as layer 1, as the
+    // running top-n with its E_sub, applies the loop test and, if the tree grows on, sends out the rows of
+    // layer 2 itself, which takes the layer team's round trip out of the first layer.  Returns false (nothing
+    // done) when layer 1 needs a selection or the tree ends with it; the layer team then does it the ordinary way.
+    __device__ bool first_layer_direct(const RowDesc& d, const RowOut& r, const SeqWork& sw) {
+        const int lane = threadIdx.x & 31;
+        const double ph = lane < r.kk ? d.pphat * r.p : 0.0;              // Eq. 2
+        const double esub = warp_sum(ph);                                  // (the order update_running_warp sums in)
+        const bool more = 1 < p.Dcap && (esub > (double)p.delta);          // loop test of Algorithm 1 with E = 0
+        if (r.kk > p.n || !more) return false;
+        const TreeOut to = tree_out(out, p, d.b);
+        unsigned g0 = 0;
+        if (lane == 0) g0 = atomicAdd(reinterpret_cast<unsigned int*>(&w.q_ctl[kQCursor]), (unsigned)r.kk);
+        g0 = __shfl_sync(0xFFFFFFFFu, g0, 0);
+        if (lane < r.kk) {
+            int token = r.tok;
+            if (token < 0 || token >= p.V) { set_status(w.status, kErrInternal); token = 0; }
+            sw.T_tok[lane] = token; sw.T_par[lane] = 0; sw.T_phat[lane] = ph;
+            sw.R[p.n + lane] = lane;                                       // the running top-n after layer 1 (buffer of odd layers)
+            if (kPrune) sw.fmap[lane] = lane;
+            const unsigned g = g0 + (unsigned)lane, c = g % (unsigned)p.grid, e = g / (unsigned)p.grid;
+            if (e < (unsigned)p.mcap) {
+                const size_t pos = (size_t)c * p.mcap + e;
+                st_relaxed_u64(&w.mb_phat[pos], phat_word(ph));
+                st_relaxed_u64(&w.mb_items[pos], item_encode(d.b, 2, lane, row_of(token, 1, p.H)));
+            } else {
+                set_status(w.status, kErrInternal);
+            }
+        }
+        if (lane == 0) {
+            if (to.esub_trace) to.esub_trace[0] = esub;
+            sw.st[kStNR] = r.kk;
+            *sw.E_prev = esub;
+        }
+        return true;
+    }
     __device__ void row_done(const RowDesc& d, const RowOut& r, FinScratch&) {
         const int lane = threadIdx.x & 31;
         const SeqWork sw = seq_work(w, p, d.b);
+        if (d.d == 1) {                                                    // the root's row
+            const bool direct = first_layer_direct(d, r, sw);
+            __syncwarp();
+            if (lane == 0) {
+                *reinterpret_cast<volatile unsigned int*>(&sw.st[kStL1]) = 0x80000000u | (direct ? (unsigned)r.kk : 0u);
+                if (direct) atom_add_relaxed_s32(&sw.st[kStDone], 1);
+            }
+            if (direct) return;
+        }
         // Candidate words validate themselves (top bit; an absent child is all ones), so neither they nor
         // the row count need a fence: the layer warp re-reads whatever it finds not yet written.
         if (lane < p.k) {
@@ -422,6 +468,17 @@ struct BuildSink {
                     done = __shfl_sync(0xFFFFFFFFu, done, 0);
                     if (done < cur_tot[q]) continue;
                     progressed = true;
+                    if (cur_d[q] == 1) {
+                        // the finisher of the root's row says whether it grew layer 1 itself (then layer 2 is on its way)
+                        unsigned int how = 0;
+                        if (lane == 0) how = poll_tok_word(reinterpret_cast<const unsigned int*>(&sw.st[kStL1]), w.status);
+                        how = __shfl_sync(0xFFFFFFFFu, how, 0) & 0x7FFFFFFFu;
+                        if (how != 0x7FFFFFFFu && how > 0) {
+                            cur_d[q] = 2; cur_f[q] = (int)how; cur_tot[q] += (int)how;
+                            if (kPrune && lane == 0) sw.st[kStRows] = cur_tot[q];
+                            continue;
+                        }
+                    }
                     const int d = cur_d[q], fsize = cur_f[q];
                     const int nvalid = fsize * p.kk, nl = nvalid < p.n ? nvalid : p.n;
                     // Without a threshold the loop test only looks at the depth: the next layer's rows

@@ -120,7 +120,8 @@ struct SeqWork {
     int32_t* st;           // [8]      1: rows finished since the build began, 2: |R|, 3: rows sent out in all
     int32_t* fmap;         // [n]      pruned draft: layer slot of the node behind each frontier row
 };
-enum { kStDone = 1, kStNR = 2, kStRows = 3, kStDepth = 4, kStFsize = 5 };   // 4, 5: layer-by-layer build: layer awaited (0: finished), its rows
+enum { kStDone = 1, kStNR = 2, kStRows = 3, kStDepth = 4, kStFsize = 5, kStL1 = 6 };   // 4, 5: layer-by-layer build: layer awaited (0: finished), its rows
+// 6: how the root's row was handled (top bit: decided; the rest: rows of layer 2 if its finisher grew layer 1 itself, else 0)
 
 struct TreeOut {           // mirrors opt_tree_out, pointers offset to the sequence
     int32_t *token, *parent, *depth;
