@@ -9,9 +9,13 @@ Everything the library computes goes through its C ABI (opt_tree_build, opt_tree
 opt_tree_row_softmax_topk).  The fixed-shape trees are the comparison, not the method: they are
 assembled here from the row step's top tokens (a complete b-ary tree cut off at n nodes, level by
 level; the sequence draft is the chain of most probable tokens, which is opt_tree_build with
-k = 1) and verified by the same opt_tree_verify.  Every shape is tried on the same root tokens:
-the decoding chain follows the adaptive tree's accepted tokens (Algorithm 2), and at every step
-the fixed trees are built and verified for that step's roots as well.
+k = 1) and verified by the same opt_tree_verify.  Every shape is tried on the same root tokens.
+Every step draws fresh seeded root tokens: the table model's whole state is the root token, so a
+chain that feeds on its own accepted tokens (Algorithm 2's Concat) falls into a cycle of a few dozen
+roots within a few steps and would sample nothing else (the parity tests follow such chains; a
+study of averages must not).  The adaptive tree is built twice: with the workload's depth limit,
+and with Algorithm 1's own limit (depth < n; here min(n, 500) layers) and threshold 0, which is
+the setting in which no tree of n nodes from the same candidates can have a larger E(A).
 """
 from __future__ import annotations
 
@@ -61,10 +65,11 @@ def _bary_tree(ot, d_ld, roots, b, n, H):
 
 
 def run(name: str, steps: int, local: int = 0, n: int | None = None, delta: float = NEG_INF, keep_first: int = 0):
-    """A free-running decoding chain of `steps` steps on workload `name` (node budget n, default the
-    workload's): acceptance length and E(A) of the adaptive tree, of the sequence draft and of the binary and
-    4-ary trees with the same number of nodes, step by step on the same roots.  keep_first: the roots of that
-    many first steps are returned too (for a check on the host)."""
+    """`steps` decoding steps on workload `name` (node budget n, default the workload's), each from fresh
+    seeded roots: acceptance length and E(A) of the adaptive tree (the workload's depth limit; and depth
+    limited by n alone with threshold 0), of the sequence draft and of the binary and 4-ary trees with the
+    same number of nodes, on the same roots.  keep_first: the roots of that many first steps are returned
+    too (for a check on the host)."""
     import torch
     from . import binding
     w = synth.WORKLOADS[name]
@@ -77,9 +82,9 @@ def run(name: str, steps: int, local: int = 0, n: int | None = None, delta: floa
     ot = binding.OptTree(w.V, w.H, n, w.k, D, B, device=dev)
     Dseq = min(n, 500)
     seq = binding.OptTree(w.V, w.H, n, 1, Dseq, B, device=dev)          # k = 1: the chain of most probable tokens
-    roots = torch.from_numpy(synth.root_tokens(B, w.V, w.seed + 1)).cuda()
-    tree, chain = ot.alloc_tree(B, trace=False), seq.alloc_tree(B, trace=False)
-    shapes = ["opt_tree", "sequence", "binary", "4-ary"]
+    deep = binding.OptTree(w.V, w.H, n, w.k, Dseq, B, device=dev)       # Algorithm 1's own depth limit
+    tree, chain, dtree = ot.alloc_tree(B, trace=False), seq.alloc_tree(B, trace=False), deep.alloc_tree(B, trace=False)
+    shapes = ["opt_tree", "opt_tree_depth_n", "sequence", "binary", "4-ary"]
     A = {s: torch.zeros((steps, B), dtype=torch.int32, device="cuda") for s in shapes}
     E = {s: torch.zeros((steps, B), dtype=torch.float64, device="cuda") for s in shapes}
     depth_of = {}
@@ -89,11 +94,16 @@ def run(name: str, steps: int, local: int = 0, n: int | None = None, delta: floa
     vs = (torch.empty(B, **i32), torch.empty((B, Dseq + 1), **i32), torch.empty((B, Dseq), **i32), torch.empty(B, **i32))
     t0 = time.perf_counter()
     for s in range(steps):
+        roots_np = synth.root_tokens(B, w.V, w.seed + 1 + s)
+        roots = torch.from_numpy(roots_np).cuda()
         if s < keep_first:
-            kept_roots.append(roots.cpu().numpy().copy())
+            kept_roots.append(roots_np.copy())
         ot.build(d_ld, roots, delta, tree)
         ot.verify(tree, d_lt, roots, vo)
         A["opt_tree"][s] = vo[0]; E["opt_tree"][s] = tree.expected_len
+        deep.build(d_ld, roots, 0.0, dtree)
+        deep.verify(dtree, d_lt, roots, vs)
+        A["opt_tree_depth_n"][s] = vs[0]; E["opt_tree_depth_n"][s] = dtree.expected_len
         seq.build(d_ld, roots, NEG_INF, chain)
         seq.verify(chain, d_lt, roots, vs)
         A["sequence"][s] = vs[0]; E["sequence"][s] = chain.expected_len
@@ -102,9 +112,8 @@ def run(name: str, steps: int, local: int = 0, n: int | None = None, delta: floa
             depth_of[shape] = lv
             fv = ot.verify(ft, d_lt, roots) if lv <= D else seq.verify(ft, d_lt, roots)
             A[shape][s] = fv[0]; E[shape][s] = ft.expected_len
-        roots = vo[3].clone()                                            # Algorithm 2: the accepted tokens extend the input
     torch.cuda.synchronize()
-    if ot.device_status() != 0 or seq.device_status() != 0:
+    if ot.device_status() != 0 or seq.device_status() != 0 or deep.device_status() != 0:
         raise RuntimeError("device status after the study")
     dt = time.perf_counter() - t0
     out = {"workload": f"{name}: batch {B}, V={w.V}, n={n}, k={w.k}, max_depth={D}, delta={'off' if delta == NEG_INF else delta}",
@@ -114,6 +123,8 @@ def run(name: str, steps: int, local: int = 0, n: int | None = None, delta: floa
         out["shapes"][s] = {"mean_acceptance_length": float(a.mean()), "mean_expected_length_plus_1": float(e.mean() + 1.0),
                             "corr_EA_A": float(np.corrcoef(a, e)[0, 1]) if a.std() > 0 and e.std() > 0 else None}
     out["shapes"]["sequence"]["depth"] = Dseq
+    out["shapes"]["opt_tree"]["depth_limit"] = D
+    out["shapes"]["opt_tree_depth_n"]["depth_limit"] = Dseq
     for s, lv in depth_of.items():
         out["shapes"][s]["depth"] = lv
     a, e = A["opt_tree"].cpu().numpy().ravel(), E["opt_tree"].cpu().numpy().ravel()
