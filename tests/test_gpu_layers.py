@@ -69,7 +69,9 @@ def test_reduced_tables(request, name, V, H, delta):
 
 
 @pytest.mark.parametrize("n,k,D,B,V", [(1, 4, 5, 3, 512), (6, 1, 6, 3, 512), (5, 8, 3, 4, 8), (7, 3, 4, 2, 12), (10, 10, 6, 5, 104),
-                                       (65, 4, 9, 2, 1024)])
+                                       (65, 4, 9, 2, 1024),
+                                       # node budgets beyond 256: the larger layout of the layer team's scratch
+                                       (300, 8, 6, 2, 2048), (1024, 32, 5, 1, 4096)])
 def test_edge_sizes(request, n, k, D, B, V):
     w = synth.Workload("edge", B, V, n, k, D, 3.0, 1.1, 0.3, H=64, seed=n * 1000 + k)
     for delta in (NEG_INF, 0.1):
