@@ -553,6 +553,7 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
         const int total = vpt << lg;
         const float negE = -(float)emax;
         float sub = 0.0f;
+        double corr = 1.0;                                  // e^gap, see below; computed while the first loads are in flight
 #pragma unroll 1
         for (int i0 = 0; i0 < total; i0 += 32 * 4) {
             uint4 w[4];
@@ -567,6 +568,12 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
                     const int vi = (j / kVecPerThread) * kChunkVecs + (j % kVecPerThread) * kConsumers + f.flist[fi];
                     if (vi < nvec) { vis[u] = vi; w[u] = load_row_vec(row, vi, V, aligned); }
                 }
+            }
+            if (i0 == 0) {
+                // Bulk terms are 2^(fl(x*L32) - E) with L32 the fp32 log2(e); wanted e^(x-m) = 2^((x-m)*L).
+                // The exponent gap E - m*L + x*(L - L32) is evaluated at a typical bulk logit x = tau - 2.
+                const double gap = (double)emax - m * kLog2eD + ((double)tau_f - 2.0) * (kLog2eD - (double)kLog2e);
+                corr = exp_f64(gap * 0.693147180559945309417);
             }
             // bit 8u+e of m32: element e of vector u is a candidate (most vectors hold none)
             uint32_t m32 = 0;
@@ -596,10 +603,7 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
         M = f.cand_count;
         if (M > 64) exact = true;
         else {
-            // Bulk terms are 2^(fl(x*L32) - E) with L32 the fp32 log2(e); wanted e^(x-m) = 2^((x-m)*L).
-            // The exponent gap E - m*L + x*(L - L32) is evaluated at a typical bulk logit x = tau - 2.
-            const double gap = (double)emax - m * kLog2eD + ((double)tau_f - 2.0) * (kLog2eD - (double)kLog2e);
-            S = warp_sum(part - (double)sub) * exp_f64(gap * 0.693147180559945309417);
+            S = warp_sum(part - (double)sub) * corr;
         }
     }
     if (exact) {
@@ -616,7 +620,7 @@ __device__ __forceinline__ void finish_row_warp(FinScratch& f, const RowSlot& sl
         const double e = lane < M ? exp_f64((double)cand_logit(mine) - m) : 0.0;
         if (!exact) S += (double)warp_sum_u64(__double2ull_rn(e * kFixScale)) / kFixScale;   // integer sum: order free
         int rank = 0;
-#pragma unroll 1
+#pragma unroll 4
         for (int j = 0; j < M; ++j) rank += __shfl_sync(0xFFFFFFFFu, mine, j) > mine ? 1 : 0;
         __syncwarp();
         if (lane < M) { f.cand[rank] = mine; f.cand[32 + rank] = (unsigned long long)__double_as_longlong(e); }

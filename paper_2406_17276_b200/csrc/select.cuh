@@ -323,6 +323,7 @@ __device__ __noinline__ int select_layer_team(LS& s, const LayerJob& j, int tt, 
     }
     int pos = team_excl_scan(gt + eq_take, s.scan_b, tw, total);
     if (dirty >= 0) { s.thist[dirty][tt] = 0; s.thist[dirty][tt + kTeam] = 0; }     // everyone is past the last pass
+    int frow = lo / j.k, frank = lo - frow * j.k;          // frontier row and sibling rank of candidate i, carried along
     #pragma unroll 1
     for (int i = lo; i < hi; ++i) {
         const unsigned long long key = s.keys[i];
@@ -333,11 +334,12 @@ __device__ __noinline__ int select_layer_team(LS& s, const LayerJob& j, int tt, 
             const int tok = t32 == ~0u ? -1 : (int)(t32 & 0x7FFFFFFFu);
             j.T_tok[gid0 + pos] = tok;
             s.ltok[pos] = tok;
-            j.T_par[gid0 + pos] = kPrune ? __ldcg(&j.fmap[i / j.k]) : i / j.k;
+            j.T_par[gid0 + pos] = kPrune ? __ldcg(&j.fmap[frow]) : frow;
             j.T_phat[gid0 + pos] = __longlong_as_double((long long)(key - 1ull));
             s.lkeys[pos] = key;
             ++pos;
         }
+        if (++frank == j.k) { frank = 0; ++frow; }
     }
     if (total != nl) set_status(status, kErrInternal);
     team_sync();
