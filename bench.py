@@ -221,6 +221,20 @@ def timed_blocks(s: Stepper, steps, warmup, delta, min_ms=MIN_TIMED_MS, max_buil
     return units / (tot_ms * 1e-3), tot_ms / (blocks * steps), blocks
 
 
+def mal_sample(s: Stepper, delta, steps=64):
+    """Mean acceptance length and mean E(A) of the workload's trees over `steps` steps from fresh seeded roots
+    (outside every timed region; a chain that follows its own accepted tokens soon cycles on these tables)."""
+    torch, w = s.torch, s.w
+    a = torch.zeros((), dtype=torch.float64, device="cuda"); e = torch.zeros((), dtype=torch.float64, device="cuda")
+    for i in range(steps):
+        s.root = torch.from_numpy(synth.root_tokens(w.batch, w.V, w.seed + 5000 + i)).cuda()
+        s.step(i, delta)
+        a += s.vout[i & 1][0].double().mean(); e += s.tree.expected_len.mean()
+    torch.cuda.synchronize()
+    return {"mean_acceptance_length": float(a) / steps, "mean_expected_length": float(e) / steps, "steps": steps,
+            "trees": steps * w.batch, "note": "A counts the bonus token, E(A) (Eq. 3) does not"}
+
+
 def quick_config(name, local, delta=NEG_INF):
     """Device-resident steps of another configuration, timed for a fraction of a second."""
     import torch
@@ -252,6 +266,7 @@ def quick_config(name, local, delta=NEG_INF):
            "frac_of_nominal_8000": gbs / 8000.0}
     if w.batch == 1:
         out["latency_ms_one_sequence"] = ms
+    out["mal"] = mal_sample(s, delta, steps=8 if name == "c5" else 64)
     del s
     torch.cuda.empty_cache()
     return out
@@ -388,6 +403,7 @@ def run_cuda(args):
     }
     if world == 1 and not args.quick:
         line.update(extras(s, args, local, rows_total))
+        line["mal"] = mal_sample(s, delta)
     del s
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
